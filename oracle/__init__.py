@@ -1,0 +1,165 @@
+"""SGEMM-cube CPU oracle: numpy front end of oracle/sgemm_cube_oracle.cpp.
+
+TEST INFRASTRUCTURE.  Nothing on the product path may import this package; it exists so that
+tests, the smoke check and the benchmark's CPU-baseline leg can compare the CUDA library with a
+slow, plain definition of the method.  It imports nothing from the CUDA package.
+
+Functions mirror the paper's steps:
+  f16_rn / f16_to_f32     FP32 <-> FP16 conversion, RN-even             [Sec. 3.3, 4.1]
+  split                   (hi, lo) two-word split with residual scale s  [Eq. recover_eqn]
+  sgemm_cube              three-product reconstruction, termwise or
+                          elementwise accumulation, k-block kb           [Eq. termwise, elementwise]
+  dgemm_ref, sgemm_f32    FP64 reference with |A||B|; plain FP32 GEMM    [Sec. 6.1]
+  frobenius_rel_err       the paper's error metric                       [Eq. err]
+  componentwise_err       max |C - C64| / (|A||B|)                       [Eq. main_bound]
+"""
+import ctypes
+import os
+
+import numpy as np
+
+from . import build as _build
+from .bounds import (U16, U32, gamma, tau, ll_coeff, main_bound_coeff,  # noqa: F401
+                     main_bound_first_order)
+
+TERMWISE = 0
+ELEMENTWISE = 1
+
+_lib = None
+
+
+def _load():
+    global _lib
+    if _lib is None:
+        path = _build.build()
+        lib = ctypes.CDLL(path)
+        i64, c_int = ctypes.c_int64, ctypes.c_int
+        vp = ctypes.c_void_p
+        lib.oracle_num_threads.restype = c_int
+        lib.oracle_f16_rn.argtypes = [ctypes.c_uint32]
+        lib.oracle_f16_rn.restype = ctypes.c_uint16
+        lib.oracle_f16_to_f32.argtypes = [ctypes.c_uint16]
+        lib.oracle_f16_to_f32.restype = ctypes.c_uint32
+        lib.oracle_f16_rn_array.argtypes = [i64, vp, vp]
+        lib.oracle_f16_rn_array.restype = None
+        lib.oracle_f16_to_f32_array.argtypes = [i64, vp, vp]
+        lib.oracle_f16_to_f32_array.restype = None
+        lib.oracle_split.argtypes = [i64, i64, vp, i64, vp, vp, i64, c_int]
+        lib.oracle_split.restype = None
+        lib.oracle_sgemm_cube.argtypes = [i64, i64, i64, vp, i64, vp, i64, vp, i64, c_int, c_int,
+                                          i64, vp, i64]
+        lib.oracle_sgemm_cube.restype = c_int
+        lib.oracle_dgemm_ref.argtypes = [i64, i64, i64, vp, i64, vp, i64, vp, vp]
+        lib.oracle_dgemm_ref.restype = None
+        lib.oracle_sgemm_f32.argtypes = [i64, i64, i64, vp, i64, vp, i64, vp, i64]
+        lib.oracle_sgemm_f32.restype = None
+        _lib = lib
+    return _lib
+
+
+def num_threads() -> int:
+    return int(_load().oracle_num_threads())
+
+
+def _f32_2d(x):
+    x = np.asarray(x)
+    if x.dtype != np.float32 or x.ndim != 2:
+        raise TypeError("expected a 2-D float32 array")
+    if x.strides[1] != 4 or x.strides[0] % 4 or x.strides[0] < 4 * x.shape[1]:
+        x = np.ascontiguousarray(x)
+    return x
+
+
+def f16_rn(bits32):
+    """FP32 bit patterns (uint32 array or int) -> FP16 bit patterns, RN-even."""
+    lib = _load()
+    if np.isscalar(bits32):
+        return int(lib.oracle_f16_rn(int(bits32) & 0xFFFFFFFF))
+    a = np.ascontiguousarray(bits32, dtype=np.uint32)
+    out = np.empty(a.shape, dtype=np.uint16)
+    lib.oracle_f16_rn_array(a.size, a.ctypes.data, out.ctypes.data)
+    return out
+
+
+def f16_to_f32(bits16):
+    """FP16 bit patterns -> FP32 bit patterns (exact)."""
+    lib = _load()
+    if np.isscalar(bits16):
+        return int(lib.oracle_f16_to_f32(int(bits16) & 0xFFFF))
+    a = np.ascontiguousarray(bits16, dtype=np.uint16)
+    out = np.empty(a.shape, dtype=np.uint32)
+    lib.oracle_f16_to_f32_array(a.size, a.ctypes.data, out.ctypes.data)
+    return out
+
+
+def split(X, s):
+    """Two-word split of a 2-D float32 array; returns (hi, lo) uint16 bit patterns."""
+    lib = _load()
+    X = _f32_2d(X)
+    rows, cols = X.shape
+    hi = np.empty((rows, cols), dtype=np.uint16)
+    lo = np.empty((rows, cols), dtype=np.uint16)
+    lib.oracle_split(rows, cols, X.ctypes.data, X.strides[0] // 4, hi.ctypes.data,
+                     lo.ctypes.data, cols, int(s))
+    return hi, lo
+
+
+def sgemm_cube(A, B, s=11, order=TERMWISE, kb=64, return_hgemm=False):
+    """C = hi_A hi_B + 2^-s (lo_A hi_B + hi_A lo_B) with FP32 accumulation in k-blocks of kb."""
+    lib = _load()
+    A, B = _f32_2d(A), _f32_2d(B)
+    M, K = A.shape
+    K2, N = B.shape
+    if K != K2:
+        raise ValueError("inner dimensions differ")
+    C = np.empty((M, N), dtype=np.float32)
+    H = np.empty((M, N), dtype=np.float32) if return_hgemm else None
+    kb = int(kb) if kb else max(K, 1)
+    rc = lib.oracle_sgemm_cube(M, N, K, A.ctypes.data, A.strides[0] // 4, B.ctypes.data,
+                               B.strides[0] // 4, C.ctypes.data, N, int(s), int(order), kb,
+                               H.ctypes.data if return_hgemm else None, N)
+    if rc != 0:
+        raise ValueError("oracle_sgemm_cube: invalid argument")
+    return (C, H) if return_hgemm else C
+
+
+def dgemm_ref(A, B, with_abs=True):
+    """(C64, |A||B|) accumulated in double."""
+    lib = _load()
+    A, B = _f32_2d(A), _f32_2d(B)
+    M, K = A.shape
+    _, N = B.shape
+    C = np.empty((M, N), dtype=np.float64)
+    AB = np.empty((M, N), dtype=np.float64) if with_abs else None
+    lib.oracle_dgemm_ref(M, N, K, A.ctypes.data, A.strides[0] // 4, B.ctypes.data,
+                         B.strides[0] // 4, C.ctypes.data, AB.ctypes.data if with_abs else None)
+    return (C, AB) if with_abs else C
+
+
+def sgemm_f32(A, B):
+    """Sequential FP32 GEMM of the unsplit inputs."""
+    lib = _load()
+    A, B = _f32_2d(A), _f32_2d(B)
+    M, K = A.shape
+    _, N = B.shape
+    C = np.empty((M, N), dtype=np.float32)
+    lib.oracle_sgemm_f32(M, N, K, A.ctypes.data, A.strides[0] // 4, B.ctypes.data,
+                         B.strides[0] // 4, C.ctypes.data, N)
+    return C
+
+
+def frobenius_rel_err(C, C64):
+    """||C_true - C||_F / ||C_true||_F  [Eq. err]."""
+    d = np.asarray(C, dtype=np.float64) - C64
+    return float(np.sqrt((d * d).sum()) / np.sqrt((C64 * C64).sum()))
+
+
+def componentwise_err(C, C64, ABabs):
+    """max_ij |C - C64| / (|A||B|)_ij; entries with (|A||B|)_ij = 0 must be exactly zero."""
+    d = np.abs(np.asarray(C, dtype=np.float64) - C64)
+    zero = ABabs == 0
+    if np.any(d[zero] != 0):
+        return float("inf")
+    if np.all(zero):
+        return 0.0
+    return float((d[~zero] / ABabs[~zero]).max())

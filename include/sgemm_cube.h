@@ -1,0 +1,177 @@
+/*
+ * sgemm_cube.h -- C ABI of the SGEMM-cube library for NVIDIA B200 (sm_100a).
+ *
+ * SGEMM-cube approximates an FP32 GEMM C = A * B (FP32 in, FP32 out) with FP16 tensor-core
+ * products.  Every FP32 operand x is split into an FP16 high word and a scaled FP16 residual,
+ *
+ *      hi = fl16(x),     lo = fl16((x - hi) * 2^s)            (round-to-nearest-even)
+ *
+ * and C is rebuilt from three FP16 x FP16 -> FP32 products, dropping lo*lo:
+ *
+ *      C  ~=  hi_A hi_B  +  2^-s ( lo_A hi_B  +  hi_A lo_B )
+ *
+ * (paper: Sec. 3.3 "FP32-to-FP16 Two-Component Representation", Eq. fp16_high_low;
+ *  Sec. 4.2 "Residual Scaling Strategy", Eq. sf_bounds; Sec. 4.3, Eq. recover_eqn;
+ *  Sec. 4.5 "Elementwise vs. Termwise Accumulation", Eq. elementwise / Eq. termwise).
+ *
+ * Conventions shared by every entry point
+ *   - All matrices are ROW-MAJOR with a leading dimension counted in elements.
+ *   - Pointers named *_dev are DEVICE pointers on the handle's device; pointers named *_host are
+ *     host pointers.  The caller owns every buffer it passes; the handle owns only its internal
+ *     workspace.  No entry point takes ownership of or frees a caller's buffer.
+ *   - `stream` is a cudaStream_t passed as void* (NULL = the default stream).  Device entry
+ *     points enqueue work on it and return without synchronising.
+ *   - Every function returns a status code (0 = success) and never throws or exits.  Argument
+ *     errors are detected before anything is enqueued.  A failure inside a kernel (a bounded
+ *     wait that ran out) is recorded in a device error word and reported by sgemm_cube_check().
+ *   - FP16 matrices are passed as uint16_t bit patterns (IEEE binary16).
+ *   - There is no CPU fallback: on a device that is not sm_100 sgemm_cube_create fails.
+ */
+#ifndef SGEMM_CUBE_H_
+#define SGEMM_CUBE_H_
+
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct sgemm_cube_ctx* sgemm_cube_handle;
+
+/* status codes */
+enum {
+  SGEMM_CUBE_OK = 0,
+  SGEMM_CUBE_INVALID_ARG = 1,      /* null pointer, non-positive size, ld too small, bad enum   */
+  SGEMM_CUBE_MISALIGNED = 2,       /* pointer / leading dimension violates an alignment rule    */
+  SGEMM_CUBE_CUDA_ERROR = 3,       /* a CUDA runtime or driver call failed                      */
+  SGEMM_CUBE_DEVICE_TIMEOUT = 4,   /* a kernel gave up on a bounded wait (see sgemm_cube_check) */
+  SGEMM_CUBE_UNSUPPORTED_ARCH = 5, /* device is not compute capability 10.x                     */
+  SGEMM_CUBE_ALLOC_FAILED = 6      /* workspace allocation failed                               */
+};
+
+/* accumulation order (paper Sec. 4.5) */
+enum {
+  SGEMM_CUBE_TERMWISE = 0,   /* Eq. termwise: streams summed separately, combined once at the end */
+  SGEMM_CUBE_ELEMENTWISE = 1 /* Eq. elementwise: per k-block, products folded into one accumulator */
+};
+
+/* options for sgemm_cube_set_option */
+enum {
+  /* Length, in k, of a chain accumulated inside the tensor core before it is added, in FP32 with
+   * round-to-nearest, to the running sum held in registers (termwise: the hi*hi stream; the
+   * correction stream is carried whole).  Multiple of 64, default 256.  This is the "k-block" g
+   * of Sec. 4.5 as realised on this hardware. */
+  SGEMM_CUBE_OPT_TERMWISE_K_BLOCK = 0,
+  /* Same for the elementwise order: the k-block of Eq. elementwise.  Multiple of 64, default 64. */
+  SGEMM_CUBE_OPT_ELEMENTWISE_K_BLOCK = 1
+};
+
+/* Create a handle bound to CUDA device `device`.  Allocates a small device error word; the
+ * workspace of the unfused path and of the host-buffer path grows on demand.
+ * Errors: INVALID_ARG (out == NULL), CUDA_ERROR, UNSUPPORTED_ARCH, ALLOC_FAILED. */
+int sgemm_cube_create(sgemm_cube_handle* out, int device);
+
+/* Synchronise the device, free the handle's workspace and the handle.  Returns DEVICE_TIMEOUT
+ * if a kernel recorded a failure that was never collected by sgemm_cube_check. */
+int sgemm_cube_destroy(sgemm_cube_handle h);
+
+/* Set an option (see SGEMM_CUBE_OPT_*).  Errors: INVALID_ARG. */
+int sgemm_cube_set_option(sgemm_cube_handle h, int option, int64_t value);
+
+/* Operand split (paper Eq. recover_eqn, first two lines; Sec. 3.3; Sec. 4.2).
+ *   hi[i,j] = fl16(X[i,j]);  lo[i,j] = fl16((X[i,j] - hi[i,j]) * 2^scale_exp)
+ * RN-even conversions; the subtraction and the scaling are exact FP32 operations; FP16
+ * subnormals are produced (gradual underflow is kept, nothing is flushed or clamped);
+ * out-of-range inputs follow IEEE (|x| >= 65520 -> hi = inf, lo = NaN or inf).
+ *   X_dev      rows x cols FP32, row-major, leading dimension ldx >= cols          (device, read)
+ *   hi_dev/lo_dev  rows x cols FP16 bit patterns, leading dimension ldh >= cols    (device, written)
+ *   scale_exp  s in [0, 24]
+ * Any alignment is accepted; 16-byte aligned pointers with ldx % 4 == 0 and ldh % 8 == 0 take
+ * the vectorised path.  Errors: INVALID_ARG, CUDA_ERROR. */
+int sgemm_cube_split(sgemm_cube_handle h, int rows, int cols,
+                     const float* X_dev, int64_t ldx,
+                     uint16_t* hi_dev, uint16_t* lo_dev, int64_t ldh,
+                     int scale_exp, void* stream);
+
+/* Fused SGEMM-cube (paper Eq. recover_eqn with Eq. termwise or Eq. elementwise):
+ *   C = hi_A hi_B + 2^-s (lo_A hi_B + hi_A lo_B),   hi/lo produced on the fly inside the kernel
+ * (no FP16 copy of A or B goes through device memory), FP16 x FP16 products on the tensor cores
+ * with FP32 accumulation, C overwritten (no alpha/beta).
+ *   A_dev  M x K FP32, lda >= K     (device, read)
+ *   B_dev  K x N FP32, ldb >= N     (device, read)
+ *   C_dev  M x N FP32, ldc >= N     (device, written)
+ *   scale_exp s in [0, 24]; accumulation_order SGEMM_CUBE_TERMWISE or SGEMM_CUBE_ELEMENTWISE
+ * Alignment: A_dev, B_dev 16-byte aligned and lda % 4 == 0, ldb % 4 == 0 (else MISALIGNED).
+ * C_dev may have any alignment.  M, N, K >= 1, any values (ragged edges are handled).
+ * Errors: INVALID_ARG, MISALIGNED, CUDA_ERROR. */
+int sgemm_cube(sgemm_cube_handle h, int M, int N, int K,
+               const float* A_dev, int64_t lda,
+               const float* B_dev, int64_t ldb,
+               float* C_dev, int64_t ldc,
+               int scale_exp, int accumulation_order, void* stream);
+
+/* Unfused ablation of the same computation (paper Sec. 5.4: one GEMM pipeline per term):
+ * split A and B into FP16 words in the handle's workspace, run three FP16 GEMM passes
+ * (hi_A hi_B -> D_hh; lo_A hi_B -> D_x; hi_A lo_B added to D_x), then C = D_hh + 2^-s D_x.
+ * Termwise only (accumulation_order must be SGEMM_CUBE_TERMWISE).  Same arguments and
+ * alignment-free inputs (the workspace copies are padded).  The workspace
+ * (4 bytes x (M K + K N) + 8 bytes x M N, rounded up) is grown with cudaMalloc on first use;
+ * Errors: INVALID_ARG, ALLOC_FAILED, CUDA_ERROR. */
+int sgemm_cube_unfused(sgemm_cube_handle h, int M, int N, int K,
+                       const float* A_dev, int64_t lda,
+                       const float* B_dev, int64_t ldb,
+                       float* C_dev, int64_t ldc,
+                       int scale_exp, int accumulation_order, void* stream);
+
+/* SGEMM-cube on operands that were split beforehand with sgemm_cube_split (all three products
+ * and the reconstruction in one kernel; useful when an operand is reused across calls).
+ *   Ahi_dev/Alo_dev  M x K FP16 bit patterns, leading dimension lda16 >= K   (device, read)
+ *   Bhi_dev/Blo_dev  K x N FP16 bit patterns, leading dimension ldb16 >= N   (device, read)
+ * Alignment: the four FP16 pointers 16-byte aligned, lda16 % 8 == 0, ldb16 % 8 == 0.
+ * scale_exp must be the value used for the split.  Errors as sgemm_cube. */
+int sgemm_cube_presplit(sgemm_cube_handle h, int M, int N, int K,
+                        const uint16_t* Ahi_dev, const uint16_t* Alo_dev, int64_t lda16,
+                        const uint16_t* Bhi_dev, const uint16_t* Blo_dev, int64_t ldb16,
+                        float* C_dev, int64_t ldc,
+                        int scale_exp, int accumulation_order, void* stream);
+
+/* Plain FP16 x FP16 -> FP32 GEMM on the tensor cores, D = A16 B16 (or D += A16 B16 when
+ * accumulate != 0): one pass of the unfused path, and the "native FP16 GEMM" the paper
+ * contrasts with (Sec. 6.2).
+ *   A16_dev M x K FP16 (lda16 >= K), B16_dev K x N FP16 (ldb16 >= N), D_dev M x N FP32 (ldd >= N).
+ * Alignment as sgemm_cube_presplit.  Errors as sgemm_cube. */
+int sgemm_cube_hgemm(sgemm_cube_handle h, int M, int N, int K,
+                     const uint16_t* A16_dev, int64_t lda16,
+                     const uint16_t* B16_dev, int64_t ldb16,
+                     float* D_dev, int64_t ldd, int accumulate, void* stream);
+
+/* Host-buffer convenience around sgemm_cube: copies A and B from HOST memory to the handle's
+ * device workspace, runs the fused kernel, copies C back to HOST memory and synchronises the
+ * stream before returning.  Pinned host memory makes the copies asynchronous to the host but the
+ * call still returns only when C_host is complete.
+ *   A_host M x K (lda >= K), B_host K x N (ldb >= N), C_host M x N (ldc >= N), all FP32 HOST.
+ * Errors: INVALID_ARG, ALLOC_FAILED, CUDA_ERROR, DEVICE_TIMEOUT. */
+int sgemm_cube_host(sgemm_cube_handle h, int M, int N, int K,
+                    const float* A_host, int64_t lda,
+                    const float* B_host, int64_t ldb,
+                    float* C_host, int64_t ldc,
+                    int scale_exp, int accumulation_order, void* stream);
+
+/* Synchronise `stream` and report (then clear) the device error word.
+ * Returns OK, DEVICE_TIMEOUT (detail in *detail_out if non-NULL: a code naming the wait that
+ * gave up) or CUDA_ERROR. */
+int sgemm_cube_check(sgemm_cube_handle h, void* stream, uint32_t* detail_out);
+
+/* Number of kernels this handle has launched since creation (for launch accounting). */
+int64_t sgemm_cube_launch_count(sgemm_cube_handle h);
+
+/* Text for a status code (static storage; never NULL). */
+const char* sgemm_cube_status_string(int status);
+
+/* Library version: major * 10000 + minor * 100 + patch. */
+int sgemm_cube_version(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* SGEMM_CUBE_H_ */

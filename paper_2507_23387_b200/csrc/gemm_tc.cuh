@@ -1,0 +1,554 @@
+// The tensor-core kernels of the library, one template:
+//
+//   <NTERMS = 1, FUSED = false> : D (+)= A16 * B16       one pass of the unfused path (Sec. 5.4:
+//                                                        "one pipeline instance per term")
+//   <NTERMS = 3, FUSED = false> : C = hi_A hi_B + 2^-s (lo_A hi_B + hi_A lo_B) from FP16 words that
+//                                 were split beforehand: all three products of Eq. recover_eqn
+//   <NTERMS = 3, FUSED = true>  : the same from the FP32 operands: converter warps split them on
+//                                 the fly (Eq. recover_eqn, first two lines), so no FP16 copy of
+//                                 A or B ever goes through device memory
+//   termwise (Eq. termwise) or elementwise (Eq. elementwise) accumulation for NTERMS == 3.
+//
+// Structure (one persistent CTA per SM):
+//   warps 0-7    accumulate/epilogue warps: tcgen05.ld the TMEM partial sums, add them with FP32
+//                round-to-nearest into running sums held in registers, form C, store it
+//   not FUSED (320 threads): warp 8 = TMA producer (FP16 tiles global -> shared, swizzled UMMA
+//                layout), warp 9 = MMA issuer
+//   FUSED (512 threads): warps 8-14 = converter warps: FP32 tiles global -> registers -> (hi, lo)
+//                FP16 words -> shared memory, written directly in the swizzled UMMA layout;
+//                warp 15 = MMA issuer.  The FP32 data never touches shared memory: with
+//                128 bytes/clk of shared-memory bandwidth per SM the tensor core's own operand
+//                reads leave no room for an FP32 staging round trip.
+//   The MMA issuer is one thread issuing tcgen05.mma kind::f16 (M = 128, N = 256, K = 16).
+//
+// Why the running sums live in registers.  The tensor core adds products into its FP32
+// accumulator without round-to-nearest, so a long chain accumulated only inside TMEM drifts
+// (the reason earlier GPU work accumulates outside the matrix unit, Sec. 4.3 last paragraph).
+// The k dimension is therefore cut into blocks g of `kchunk` elements (the k-blocks of Sec. 4.5);
+// each block's product is accumulated in TMEM from zero and then added, with an IEEE RN FP32
+// addition, to the register-resident sum.  For the termwise order only the dominant hi*hi stream
+// needs this; the correction stream (scaled by 2^-s at the end) is carried in TMEM for the whole k.
+//
+// TMEM: 512 columns = two regions of 256 columns (one 128 x 256 FP32 tile each).
+//   NTERMS == 1             : the regions alternate between consecutive k-blocks (double buffer)
+//   NTERMS == 3 termwise    : R0 = hi*hi partial of the current k-block, R1 = correction stream
+//   NTERMS == 3 elementwise : R0 = hi*hi partial, R1 = correction partial of the current k-block
+#pragma once
+
+#include <cuda_fp16.h>
+
+#include "ptx_sm100.cuh"
+
+namespace sgc {
+
+constexpr int kBM = 128;            // CTA tile rows  (UMMA M)
+constexpr int kBN = 256;            // CTA tile cols  (UMMA N)
+constexpr int kNumEpiWarps = 8;     // warps 0-7
+constexpr int kTcThreads = 320;     // not FUSED: + TMA warp + MMA warp
+constexpr int kFusedThreads = 512;  // FUSED: + 7 converter warps + MMA warp
+constexpr int kNumConvWarps = 7;
+constexpr int kConvThreads = kNumConvWarps * 32;   // 224
+constexpr uint32_t kTmemCols = 512;
+
+// error codes written to the device error word (which wait gave up)
+enum : unsigned int {
+  kErrProducerEmptyWait = 0x101,
+  kErrMmaFullWait = 0x102,
+  kErrMmaTmemEmptyWait = 0x103,
+  kErrEpiTmemFullWait = 0x104,
+  kErrDrainWait = 0x105,
+  kErrConvEmptyWait = 0x106,
+};
+
+struct TcGemmParams {
+  int M, N, K;
+  float* D;             // output (C for NTERMS == 3)
+  long long ldd;
+  int accumulate;       // NTERMS == 1 only: D += result
+  int order;            // NTERMS == 3: 0 termwise, 1 elementwise
+  int kchunk_blocks;    // k-block length in units of the stage depth BK
+  float inv_scale;      // 2^-s
+  unsigned int* err;    // device error word
+  // FUSED only: the FP32 operands (row-major, 16-byte aligned, leading dimensions % 4 == 0)
+  const float* A32;
+  long long lda32;
+  const float* B32;
+  long long ldb32;
+  float scale;          // 2^s
+};
+
+template <int NTERMS>
+struct TcCfg {
+  static constexpr int BK = (NTERMS == 1) ? 64 : 32;      // k per pipeline stage
+  static constexpr int STAGES = 4;
+  static constexpr int A_ROW_BYTES = BK * 2;              // 128 or 64: also the swizzle span of A
+  static constexpr uint32_t A_TILE = kBM * BK * 2;        // one FP16 A tile
+  static constexpr uint32_t B_TILE = BK * kBN * 2;        // one FP16 B tile
+  static constexpr uint32_t STAGE_BYTES = (NTERMS == 1) ? (A_TILE + B_TILE) : 2 * (A_TILE + B_TILE);
+  static constexpr uint32_t SMEM_BYTES = STAGES * STAGE_BYTES + 1024 /*align*/ + 256 /*barriers*/;
+};
+
+// Tile rasterisation: groups of 8 tile-rows are walked column by column so that the CTAs
+// running at the same time share A and B tiles in L2.
+__device__ __forceinline__ void tile_coords(int tile, int num_m, int num_n, int& tm, int& tn) {
+  constexpr int kGroupM = 8;
+  const int per_group = kGroupM * num_n;
+  const int group = tile / per_group;
+  const int first_m = group * kGroupM;
+  const int gsz = min(num_m - first_m, kGroupM);
+  const int in_group = tile - group * per_group;
+  tm = first_m + in_group % gsz;
+  tn = in_group / gsz;
+}
+
+// Epilogue helper: thread-owned row `row`, columns [col0, col0 + 16) of the output.
+__device__ __forceinline__ void store16(float* D, long long ldd, int M, int N, int row, int col0,
+                                        const float* v, bool vec_ok, int accumulate) {
+  if (row >= M || col0 >= N) return;
+  float* p = D + (long long)row * ldd + col0;
+  if (vec_ok && col0 + 16 <= N) {
+#pragma unroll
+    for (int q = 0; q < 4; ++q) {
+      float4 o = make_float4(v[4 * q], v[4 * q + 1], v[4 * q + 2], v[4 * q + 3]);
+      if (accumulate) {
+        const float4 old = *reinterpret_cast<const float4*>(p + 4 * q);
+        o.x = __fadd_rn(old.x, o.x); o.y = __fadd_rn(old.y, o.y);
+        o.z = __fadd_rn(old.z, o.z); o.w = __fadd_rn(old.w, o.w);
+      }
+      *reinterpret_cast<float4*>(p + 4 * q) = o;
+    }
+  } else {
+#pragma unroll
+    for (int j = 0; j < 16; ++j)
+      if (col0 + j < N) p[j] = accumulate ? __fadd_rn(p[j], v[j]) : v[j];
+  }
+}
+
+// ------------------------------------------------------------------------------------------
+// Converter-warp helpers (FUSED).  One "item" is 8 consecutive FP32 elements of a row (32 bytes
+// in, one 16-byte chunk of the hi tile and one of the lo tile out).
+struct ConvItem { float4 a, b; };
+
+__device__ __forceinline__ void split_pair(float x0, float x1, float scale, uint32_t& hi2,
+                                           uint32_t& lo2) {
+  // hi = fl16(x); lo = fl16((x - hi) * 2^s): the subtraction and the scaling are exact (Sec. 3.3).
+  const __half2 h = __floats2half2_rn(x0, x1);
+  const float2 hf = __half22float2(h);
+  const __half2 l = __floats2half2_rn(__fmul_rn(__fsub_rn(x0, hf.x), scale),
+                                      __fmul_rn(__fsub_rn(x1, hf.y), scale));
+  hi2 = *reinterpret_cast<const uint32_t*>(&h);
+  lo2 = *reinterpret_cast<const uint32_t*>(&l);
+}
+
+__device__ __forceinline__ void convert_store(const ConvItem& it, float scale, uint32_t hi_addr,
+                                              uint32_t lo_addr) {
+  uint4 h, l;
+  split_pair(it.a.x, it.a.y, scale, h.x, l.x);
+  split_pair(it.a.z, it.a.w, scale, h.y, l.y);
+  split_pair(it.b.x, it.b.y, scale, h.z, l.z);
+  split_pair(it.b.z, it.b.w, scale, h.w, l.w);
+  asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(hi_addr), "r"(h.x), "r"(h.y),
+               "r"(h.z), "r"(h.w) : "memory");
+  asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(lo_addr), "r"(l.x), "r"(l.y),
+               "r"(l.z), "r"(l.w) : "memory");
+}
+
+// 8 elements of row `row` starting at column `col` of a rows x cols row-major matrix; elements
+// outside the matrix read as zero (split(0) = (0, 0), so zero padding is exact).
+__device__ __forceinline__ ConvItem load_item_guarded(const float* __restrict__ X, long long ld,
+                                                      int rows, int cols, int row, int col) {
+  ConvItem it;
+  if (row < rows && col + 8 <= cols) {
+    const float4* src = reinterpret_cast<const float4*>(X + (long long)row * ld + col);
+    it.a = __ldg(src);
+    it.b = __ldg(src + 1);
+  } else {
+    float v[8];
+#pragma unroll
+    for (int j = 0; j < 8; ++j)
+      v[j] = (row < rows && col + j < cols) ? __ldg(X + (long long)row * ld + col + j) : 0.f;
+    it.a = make_float4(v[0], v[1], v[2], v[3]);
+    it.b = make_float4(v[4], v[5], v[6], v[7]);
+  }
+  return it;
+}
+
+template <int NTERMS, bool FUSED>
+__global__ void __launch_bounds__(FUSED ? kFusedThreads : kTcThreads, 1)
+tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA0, const __grid_constant__ CUtensorMap tmA1,
+               const __grid_constant__ CUtensorMap tmB0, const __grid_constant__ CUtensorMap tmB1,
+               const TcGemmParams p) {
+  using Cfg = TcCfg<NTERMS>;
+  constexpr int BK = Cfg::BK;
+  constexpr int STAGES = Cfg::STAGES;
+  constexpr int kProducerWarp = 8;                    // not FUSED
+  constexpr int kMmaWarp = FUSED ? 15 : 9;
+  static_assert(!FUSED || NTERMS == 3, "the fused kernel computes all three products");
+
+  extern __shared__ uint8_t smem_raw[];
+  // 1024-byte alignment: the swizzle pattern of TMA and of the UMMA descriptors is a function
+  // of the shared-memory address bits, so every tile must start on a 1024-byte boundary.
+  uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) &
+                                             ~uintptr_t(1023));
+  uint64_t* bars = reinterpret_cast<uint64_t*>(smem + STAGES * Cfg::STAGE_BYTES);
+  uint64_t* full_bar = bars;                 // [STAGES]  producer/converters -> MMA
+  uint64_t* empty_bar = bars + STAGES;       // [STAGES]  MMA -> producer/converters
+  uint64_t* tfull_bar = bars + 2 * STAGES;   // [2]       MMA -> epilogue (TMEM region filled)
+  uint64_t* tempty_bar = bars + 2 * STAGES + 2;  // [2]   epilogue -> MMA (TMEM region drained)
+  uint64_t* drain_bar = bars + 2 * STAGES + 4;   // [1]
+  uint32_t* tmem_base_slot = reinterpret_cast<uint32_t*>(bars + 2 * STAGES + 5);
+  volatile uint32_t* abort_flag = tmem_base_slot + 1;
+
+  const int warp = threadIdx.x >> 5;
+  const int lane = threadIdx.x & 31;
+
+  if (threadIdx.x == 0) {
+    for (int s = 0; s < STAGES; ++s) {
+      mbar_init(&full_bar[s], FUSED ? kNumConvWarps : 1);
+      mbar_init(&empty_bar[s], 1);
+    }
+    for (int r = 0; r < 2; ++r) { mbar_init(&tfull_bar[r], 1); mbar_init(&tempty_bar[r], kNumEpiWarps); }
+    mbar_init(drain_bar, 1);
+    *abort_flag = 0u;
+    fence_mbar_init();
+  }
+  if (!FUSED && warp == kProducerWarp && lane == 0) {
+    tma_prefetch_desc(&tmA0); tma_prefetch_desc(&tmB0);
+    if (NTERMS == 3) { tma_prefetch_desc(&tmA1); tma_prefetch_desc(&tmB1); }
+  }
+  if (warp == kMmaWarp) {    // whole warp: allocate all 512 TMEM columns
+    tmem_alloc(tmem_base_slot, kTmemCols);
+    tmem_relinquish();
+  }
+  tc_fence_before_sync();
+  __syncthreads();
+  tc_fence_after_sync();
+  const uint32_t tmem_base = *tmem_base_slot;
+
+  const int num_m = (p.M + kBM - 1) / kBM;
+  const int num_n = (p.N + kBN - 1) / kBN;
+  const int num_tiles = num_m * num_n;
+  const int num_kb = (p.K + BK - 1) / BK;                      // pipeline stages per tile
+  const int chunk = p.kchunk_blocks;                           // stages per k-block g
+  const int num_chunks = (num_kb + chunk - 1) / chunk;
+
+  // Register budget when FUSED (512 threads x 128 registers): the accumulate warps hold a
+  // 128 x 256 FP32 tile in registers, so warpgroups 2-3 hand registers over to warpgroups 0-1
+  // (256 x 168 + 256 x 88 = 65536).  Each setmaxnreg sits at the top of its role's branch so
+  // that the code below it is compiled against the new limit.
+  if (warp < kNumEpiWarps) {
+    if (FUSED) setmaxnreg_inc<168>();
+    // ------------------------------------------------------------------ accumulate / epilogue
+    const int quarter = warp & 3;                 // TMEM lanes 32*quarter .. +31 (warp id mod 4)
+    const int half = warp >> 2;                   // columns [128*half, 128*half + 128)
+    const uint32_t lane_addr = (uint32_t)(quarter * 32) << 16;
+    const bool vec_ok = ((reinterpret_cast<uintptr_t>(p.D) & 15) == 0) && ((p.ldd & 3) == 0);
+    uint32_t drains[2] = {0, 0};
+    uint32_t gchunk = 0;
+    bool ok = true;
+    float S[128];
+    for (int tile = blockIdx.x; tile < num_tiles && ok; tile += gridDim.x) {
+      int tm, tn;
+      tile_coords(tile, num_m, num_n, tm, tn);
+      for (int c = 0; c < num_chunks && ok; ++c, ++gchunk) {
+        const int r_main = (NTERMS == 1) ? (int)(gchunk & 1) : 0;
+        const bool with_x = (NTERMS == 3) && (p.order == 1);
+        if (!mbar_wait_bounded(&tfull_bar[r_main], drains[r_main] & 1, abort_flag, p.err,
+                               kErrEpiTmemFullWait)) { ok = false; break; }
+        if (with_x && !mbar_wait_bounded(&tfull_bar[1], drains[1] & 1, abort_flag, p.err,
+                                         kErrEpiTmemFullWait)) { ok = false; break; }
+        tc_fence_after_sync();
+        const uint32_t t_main = tmem_base + lane_addr + r_main * kBN + half * 128;
+        const uint32_t t_x = tmem_base + lane_addr + kBN + half * 128;
+#pragma unroll
+        for (int g = 0; g < 8; ++g) {
+          uint32_t v[16];
+          tmem_ld_32x32b_x16(t_main + g * 16, v);
+          tmem_ld_wait();
+          if (c == 0) {
+#pragma unroll
+            for (int j = 0; j < 16; ++j) S[g * 16 + j] = __uint_as_float(v[j]);
+          } else {
+#pragma unroll
+            for (int j = 0; j < 16; ++j) S[g * 16 + j] = __fadd_rn(S[g * 16 + j], __uint_as_float(v[j]));
+          }
+          if (with_x) {
+            // Elementwise: fold this k-block's corrections into the same accumulator.
+            tmem_ld_32x32b_x16(t_x + g * 16, v);
+            tmem_ld_wait();
+#pragma unroll
+            for (int j = 0; j < 16; ++j)
+              S[g * 16 + j] = __fadd_rn(S[g * 16 + j], __fmul_rn(__uint_as_float(v[j]), p.inv_scale));
+          }
+        }
+        tc_fence_before_sync();
+        __syncwarp();
+        if (lane == 0) {
+          mbar_arrive(&tempty_bar[r_main]);
+          if (with_x) mbar_arrive(&tempty_bar[1]);
+        }
+        drains[r_main]++;
+        if (with_x) drains[1]++;
+      }
+      if (!ok) break;
+      const int row = tm * kBM + quarter * 32 + lane;
+      const int col_base = tn * kBN + half * 128;
+      if (NTERMS == 3 && p.order == 0) {
+        // Termwise: the correction stream meets the dominant stream once, here.
+        if (!mbar_wait_bounded(&tfull_bar[1], drains[1] & 1, abort_flag, p.err, kErrEpiTmemFullWait)) {
+          ok = false;
+          break;
+        }
+        tc_fence_after_sync();
+        const uint32_t t_x = tmem_base + lane_addr + kBN + half * 128;
+#pragma unroll
+        for (int g = 0; g < 8; ++g) {
+          uint32_t v[16];
+          tmem_ld_32x32b_x16(t_x + g * 16, v);
+          tmem_ld_wait();
+#pragma unroll
+          for (int j = 0; j < 16; ++j)
+            S[g * 16 + j] = __fadd_rn(S[g * 16 + j], __fmul_rn(__uint_as_float(v[j]), p.inv_scale));
+        }
+        tc_fence_before_sync();
+        __syncwarp();
+        if (lane == 0) mbar_arrive(&tempty_bar[1]);
+        drains[1]++;
+      }
+#pragma unroll
+      for (int g = 0; g < 8; ++g)
+        store16(p.D, p.ldd, p.M, p.N, row, col_base + g * 16, &S[g * 16], vec_ok,
+                (NTERMS == 1) ? p.accumulate : 0);
+    }
+  } else if (warp == kMmaWarp) {
+    if (FUSED) setmaxnreg_dec<88>();
+    // ------------------------------------------------------------------ MMA issuer
+    if (lane == 0) {
+      constexpr uint32_t idesc = umma_idesc_f16(kBM, kBN, /*A MN-major*/ false, /*B MN-major*/ true);
+      constexpr uint64_t a_swz = (Cfg::A_ROW_BYTES == 128) ? kSwizzle128 : kSwizzle64;
+      constexpr uint32_t a_sbo = 8 * Cfg::A_ROW_BYTES;     // 8 rows of the swizzle atom
+      constexpr uint32_t b_lbo = BK * 128;                 // next 64-column atom of B
+      constexpr uint32_t b_sbo = 1024;                     // next 8 k-rows inside an atom
+      uint32_t it = 0;
+      uint32_t fills[2] = {0, 0};     // how many times each TMEM region has been handed over
+      uint32_t gchunk = 0;            // running k-block counter (NTERMS == 1 region choice)
+      bool ok = true;
+      for (int tile = blockIdx.x; tile < num_tiles && ok; tile += gridDim.x) {
+        for (int c = 0; c < num_chunks && ok; ++c, ++gchunk) {
+          const int kb_begin = c * chunk;
+          const int kb_end = min(num_kb, kb_begin + chunk);
+          // Region(s) this k-block accumulates into, and which of them start from zero here.
+          const int r_main = (NTERMS == 1) ? (int)(gchunk & 1) : 0;
+          const bool x_fresh = (NTERMS == 3) && (p.order == 1 || c == 0);
+          bool main_ready = false, x_ready = !x_fresh;
+          for (int kb = kb_begin; kb < kb_end && ok; ++kb, ++it) {
+            const int s = it % STAGES;
+            const uint32_t ph = (it / STAGES) & 1;
+            if (!mbar_wait_bounded(&full_bar[s], ph, abort_flag, p.err, kErrMmaFullWait)) {
+              ok = false;
+              break;
+            }
+            tc_fence_after_sync();
+            const uint32_t st = smem_u32(smem + s * Cfg::STAGE_BYTES);
+            const uint32_t a_hi = st;
+            const uint32_t a_lo = st + Cfg::A_TILE;
+            const uint32_t b_hi = st + ((NTERMS == 3) ? 2 * Cfg::A_TILE : Cfg::A_TILE);
+            const uint32_t b_lo = b_hi + Cfg::B_TILE;
+            const bool first_kb = (kb == kb_begin);
+            if (NTERMS == 3) {
+              // Correction products first: they do not depend on region 0 being drained, so the
+              // accumulate warps get this time to add the previous k-block into their sums.
+              if (!x_ready) {
+                if (!mbar_wait_bounded(&tempty_bar[1], (fills[1] & 1) ^ 1, abort_flag, p.err,
+                                       kErrMmaTmemEmptyWait)) { ok = false; break; }
+                tc_fence_after_sync();
+                x_ready = true;
+              }
+              const uint32_t d_x = tmem_base + kBN;
+#pragma unroll
+              for (int j = 0; j < BK / 16; ++j) {
+                const uint64_t da = umma_smem_desc(a_lo + j * 32, 16, a_sbo, a_swz);
+                const uint64_t db = umma_smem_desc(b_hi + j * 2048, b_lbo, b_sbo, kSwizzle128);
+                umma_f16_ss(d_x, da, db, idesc, (x_fresh && first_kb && j == 0) ? 0u : 1u);
+              }
+#pragma unroll
+              for (int j = 0; j < BK / 16; ++j) {
+                const uint64_t da = umma_smem_desc(a_hi + j * 32, 16, a_sbo, a_swz);
+                const uint64_t db = umma_smem_desc(b_lo + j * 2048, b_lbo, b_sbo, kSwizzle128);
+                umma_f16_ss(d_x, da, db, idesc, 1u);
+              }
+            }
+            if (!main_ready) {
+              if (!mbar_wait_bounded(&tempty_bar[r_main], (fills[r_main] & 1) ^ 1, abort_flag, p.err,
+                                     kErrMmaTmemEmptyWait)) { ok = false; break; }
+              tc_fence_after_sync();
+              main_ready = true;
+            }
+            const uint32_t d_main = tmem_base + r_main * kBN;
+#pragma unroll
+            for (int j = 0; j < BK / 16; ++j) {
+              const uint64_t da = umma_smem_desc(a_hi + j * 32, 16, a_sbo, a_swz);
+              const uint64_t db = umma_smem_desc(b_hi + j * 2048, b_lbo, b_sbo, kSwizzle128);
+              umma_f16_ss(d_main, da, db, idesc, (first_kb && j == 0) ? 0u : 1u);
+            }
+            umma_commit(&empty_bar[s]);          // stage s may be refilled once these MMAs retire
+          }
+          if (!ok) break;
+          // Hand the finished region(s) to the accumulate warps.
+          umma_commit(&tfull_bar[r_main]);
+          fills[r_main]++;
+          if (NTERMS == 3 && (p.order == 1 || c == num_chunks - 1)) {
+            umma_commit(&tfull_bar[1]);
+            fills[1]++;
+          }
+        }
+      }
+      // Bounded drain: all issued MMAs must have retired before TMEM is freed.
+      umma_commit(drain_bar);
+      mbar_wait_bounded(drain_bar, 0, nullptr, p.err, kErrDrainWait);
+    }
+  } else if (!FUSED) {
+    // ------------------------------------------------------------------ TMA producer (warp 8)
+    if (lane == 0) {
+      uint32_t it = 0;
+      bool ok = true;
+      for (int tile = blockIdx.x; tile < num_tiles && ok; tile += gridDim.x) {
+        int tm, tn;
+        tile_coords(tile, num_m, num_n, tm, tn);
+        for (int kb = 0; kb < num_kb; ++kb, ++it) {
+          const int s = it % STAGES;
+          const uint32_t ph = (it / STAGES) & 1;
+          if (!mbar_wait_bounded(&empty_bar[s], ph ^ 1, abort_flag, p.err, kErrProducerEmptyWait)) {
+            ok = false;
+            break;
+          }
+          uint8_t* st = smem + s * Cfg::STAGE_BYTES;
+          mbar_arrive_expect_tx(&full_bar[s], Cfg::STAGE_BYTES);
+          const int k0 = kb * BK;
+          // A tiles: box {BK (k), 128 rows}.  B tiles: 4 boxes {64 (n), BK (k rows)}.
+          tma_load_2d(st, &tmA0, k0, tm * kBM, &full_bar[s]);
+          uint8_t* bdst = st + Cfg::A_TILE;
+          if (NTERMS == 3) {
+            tma_load_2d(st + Cfg::A_TILE, &tmA1, k0, tm * kBM, &full_bar[s]);
+            bdst = st + 2 * Cfg::A_TILE;
+          }
+#pragma unroll
+          for (int a = 0; a < kBN / 64; ++a)
+            tma_load_2d(bdst + a * (BK * 128), &tmB0, tn * kBN + a * 64, k0, &full_bar[s]);
+          if (NTERMS == 3) {
+#pragma unroll
+            for (int a = 0; a < kBN / 64; ++a)
+              tma_load_2d(bdst + Cfg::B_TILE + a * (BK * 128), &tmB1, tn * kBN + a * 64, k0,
+                          &full_bar[s]);
+          }
+        }
+      }
+      // Bounded drain: wait until the consumer has released every stage that was filled, so
+      // that no bulk copy is in flight when the CTA exits.
+      if (ok) {
+        for (int d = 0; d < STAGES && d < (int)it; ++d, ++it) {
+          const int s = it % STAGES;
+          const uint32_t ph = (it / STAGES) & 1;
+          if (!mbar_wait_bounded(&empty_bar[s], ph ^ 1, abort_flag, p.err, kErrDrainWait)) break;
+        }
+      }
+    }
+  } else {
+    setmaxnreg_dec<88>();
+    // ------------------------------------------------------------------ converter warps (8-14)
+    // Per stage: A tile 128 x 32 FP32 = 512 items (ids 0-511: row m = id / 4, chunk q = id % 4 of
+    // 8 k), B tile 32 x 256 FP32 = 1024 items (ids 512-1535: k-row = (id - 512) / 32, chunk c of
+    // 8 n).  Thread t of the 224 takes ids t, t + 224, ..., t + 6 * 224 (the last round is partly
+    // idle).  A warp's 32 items are 8 rows x 128 bytes of A or one k-row x 1024 bytes of B:
+    // coalesced loads and bank-conflict-free 16-byte stores into the swizzled tiles.
+    //   A item -> byte offset m * 64 + ((q ^ ((m >> 1) & 3)) << 4) in the hi/lo A tile (64-byte swizzle)
+    //   B item -> atom (c / 8) * 4096 + k * 128 + (((c % 8) ^ (k % 8)) << 4) in the hi/lo B tile
+    constexpr int kRounds = 7;
+    constexpr uint32_t kInvalid = 0xFFFFFFFFu;
+    const int ct = threadIdx.x - kNumEpiWarps * 32;
+    uint32_t soff[kRounds];     // byte offset of the item's hi chunk inside the stage
+    uint32_t goff[kRounds];     // element offset of the item from the tile's first element
+#pragma unroll
+    for (int r = 0; r < kRounds; ++r) {
+      const int id = ct + r * kConvThreads;
+      if (id < 512) {
+        const int m = id >> 2, q = id & 3;
+        soff[r] = (uint32_t)(m * 64 + ((q ^ ((m >> 1) & 3)) << 4));
+        goff[r] = (uint32_t)(m * (int)p.lda32 + q * 8);
+      } else if (id < 1536) {
+        const int b = id - 512, k = b >> 5, c = b & 31;
+        soff[r] = 2 * Cfg::A_TILE + (uint32_t)((c >> 3) * (BK * 128) + k * 128 + (((c & 7) ^ (k & 7)) << 4));
+        goff[r] = (uint32_t)(k * (int)p.ldb32 + c * 8);
+      } else {
+        soff[r] = kInvalid;
+        goff[r] = 0;
+      }
+    }
+    const int total_stages = ((num_tiles - (int)blockIdx.x + (int)gridDim.x - 1) / (int)gridDim.x) * num_kb;
+    ConvItem item[kRounds];
+    // Coordinates of the stage whose FP32 data is being loaded (one stage ahead of conversion).
+    int ld_tile = blockIdx.x, ld_kb = 0, ld_tm = 0, ld_tn = 0;
+    if (ld_tile < num_tiles) tile_coords(ld_tile, num_m, num_n, ld_tm, ld_tn);
+    auto load_round = [&](int r) {
+      const int id = ct + r * kConvThreads;
+      const int m0 = ld_tm * kBM, n0 = ld_tn * kBN, k0 = ld_kb * BK;
+      const bool interior = (m0 + kBM <= p.M) && (n0 + kBN <= p.N) && (k0 + BK <= p.K);
+      if (soff[r] == kInvalid) return;
+      const bool is_a = id < 512;
+      if (interior) {
+        const float* org = is_a ? (p.A32 + (long long)m0 * p.lda32 + k0)
+                                : (p.B32 + (long long)k0 * p.ldb32 + n0);
+        const float4* src = reinterpret_cast<const float4*>(org + goff[r]);
+        item[r].a = __ldg(src);
+        item[r].b = __ldg(src + 1);
+      } else if (is_a) {
+        item[r] = load_item_guarded(p.A32, p.lda32, p.M, p.K, m0 + (id >> 2), k0 + (id & 3) * 8);
+      } else {
+        const int b = id - 512;
+        item[r] = load_item_guarded(p.B32, p.ldb32, p.K, p.N, k0 + (b >> 5), n0 + (b & 31) * 8);
+      }
+    };
+    if (total_stages > 0) {
+#pragma unroll
+      for (int r = 0; r < kRounds; ++r) load_round(r);
+    }
+    for (int it = 0; it < total_stages; ++it) {
+      const int s = it % STAGES;
+      const uint32_t ph = (it / STAGES) & 1;
+      // advance the load coordinates to stage it + 1
+      if (++ld_kb == num_kb) {
+        ld_kb = 0;
+        ld_tile += gridDim.x;
+        if (ld_tile < num_tiles) tile_coords(ld_tile, num_m, num_n, ld_tm, ld_tn);
+      }
+      const bool more = (it + 1 < total_stages);
+      if (!mbar_wait_bounded(&empty_bar[s], ph ^ 1, abort_flag, p.err, kErrConvEmptyWait)) break;
+      const uint32_t st = smem_u32(smem + s * Cfg::STAGE_BYTES);
+      // Convert the items loaded one stage ago; reload each register set as soon as it is free,
+      // so that about one stage of FP32 data per thread is always in flight.
+#pragma unroll
+      for (int r = 0; r < kRounds; ++r) {
+        if (soff[r] != kInvalid) {
+          const uint32_t lo_delta = (ct + r * kConvThreads < 512) ? Cfg::A_TILE : Cfg::B_TILE;
+          convert_store(item[r], p.scale, st + soff[r], st + soff[r] + lo_delta);
+          if (more) load_round(r);
+        }
+      }
+      // Generic-proxy stores must be visible to the tensor core (async proxy) before the hand-over.
+      fence_proxy_async_smem();
+      __syncwarp();
+      if (lane == 0) mbar_arrive(&full_bar[s]);
+    }
+  }
+
+  // ---------------------------------------------------------------------- teardown
+  tc_fence_before_sync();
+  __syncthreads();
+  if (warp == kMmaWarp) {
+    __syncwarp();
+    tc_fence_after_sync();
+    tmem_dealloc(tmem_base, kTmemCols);
+  }
+}
+
+}  // namespace sgc

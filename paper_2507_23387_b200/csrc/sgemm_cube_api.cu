@@ -1,0 +1,429 @@
+// C ABI of the SGEMM-cube library (declarations and contracts: include/sgemm_cube.h).
+// Host side only validates arguments, builds TMA descriptors and launches; every step of the
+// computation runs in the kernels of this directory.
+#include <cstdio>
+#include <cstdlib>
+#include <cstring>
+#include <new>
+
+#include <cuda.h>
+#include <cuda_runtime.h>
+
+#include "../../include/sgemm_cube.h"
+#include "gemm_tc.cuh"
+#include "split_kernel.cuh"
+
+namespace {
+
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*,
+                                  const cuuint64_t*, const cuuint64_t*, const cuuint32_t*,
+                                  const cuuint32_t*, CUtensorMapInterleave, CUtensorMapSwizzle,
+                                  CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+struct DeviceGuard {
+  int prev = -1;
+  bool ok = true;
+  explicit DeviceGuard(int dev) {
+    if (cudaGetDevice(&prev) != cudaSuccess) { ok = false; return; }
+    if (prev != dev && cudaSetDevice(dev) != cudaSuccess) ok = false;
+  }
+  ~DeviceGuard() {
+    if (prev >= 0) cudaSetDevice(prev);
+  }
+};
+
+inline size_t round_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
+inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+}  // namespace
+
+struct sgemm_cube_ctx {
+  int device = 0;
+  int sm_count = 0;
+  unsigned int* err_dev = nullptr;
+  void* ws = nullptr;          // unfused path: FP16 words of A and B, D_hh, D_x
+  size_t ws_bytes = 0;
+  void* host_ws = nullptr;     // host-buffer path: device copies of A, B, C
+  size_t host_ws_bytes = 0;
+  long long launches = 0;
+  int kblock_termwise = 256;
+  int kblock_elementwise = 64;
+  EncodeTiledFn encode = nullptr;
+  bool attrs_set = false;
+};
+
+namespace {
+
+int grow(void** buf, size_t* have, size_t want) {
+  if (*have >= want) return SGEMM_CUBE_OK;
+  if (*buf) {
+    if (cudaFree(*buf) != cudaSuccess) return SGEMM_CUBE_CUDA_ERROR;
+    *buf = nullptr;
+    *have = 0;
+  }
+  if (cudaMalloc(buf, want) != cudaSuccess) {
+    cudaGetLastError();
+    *buf = nullptr;
+    return SGEMM_CUBE_ALLOC_FAILED;
+  }
+  *have = want;
+  return SGEMM_CUBE_OK;
+}
+
+// 2-D tensor map over a row-major matrix: dims {inner, outer}, row pitch in bytes.
+int make_map(sgemm_cube_ctx* h, CUtensorMap* map, CUtensorMapDataType dt, size_t elem, const void* base,
+             uint64_t inner, uint64_t outer, uint64_t ld_elems, uint32_t box_inner,
+             uint32_t box_outer, CUtensorMapSwizzle swz) {
+  cuuint64_t dims[2] = {inner, outer};
+  cuuint64_t strides[1] = {ld_elems * elem};
+  cuuint32_t box[2] = {box_inner, box_outer};
+  cuuint32_t estr[2] = {1, 1};
+  CUresult r = h->encode(map, dt, 2, const_cast<void*>(base), dims, strides, box, estr,
+                         CU_TENSOR_MAP_INTERLEAVE_NONE, swz, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                         CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  return r == CUDA_SUCCESS ? SGEMM_CUBE_OK : SGEMM_CUBE_CUDA_ERROR;
+}
+
+int set_kernel_attrs(sgemm_cube_ctx* h) {
+  if (h->attrs_set) return SGEMM_CUBE_OK;
+  if (cudaFuncSetAttribute(sgc::tc_gemm_kernel<1, false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                           (int)sgc::TcCfg<1>::SMEM_BYTES) != cudaSuccess ||
+      cudaFuncSetAttribute(sgc::tc_gemm_kernel<3, false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                           (int)sgc::TcCfg<3>::SMEM_BYTES) != cudaSuccess ||
+      cudaFuncSetAttribute(sgc::tc_gemm_kernel<3, true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                           (int)sgc::TcCfg<3>::SMEM_BYTES) != cudaSuccess) {
+    cudaGetLastError();
+    return SGEMM_CUBE_CUDA_ERROR;
+  }
+  h->attrs_set = true;
+  return SGEMM_CUBE_OK;
+}
+
+int check_gemm_dims(int M, int N, int K, int64_t lda, int64_t ldb, int64_t ldc) {
+  if (M <= 0 || N <= 0 || K <= 0) return SGEMM_CUBE_INVALID_ARG;
+  if (lda < K || ldb < N || ldc < N) return SGEMM_CUBE_INVALID_ARG;
+  return SGEMM_CUBE_OK;
+}
+
+int launch_split(sgemm_cube_ctx* h, int rows, int cols, const float* X, int64_t ldx, uint16_t* hi,
+                 uint16_t* lo, int64_t ldh, int s, cudaStream_t st) {
+  const bool vec = (cols % 8 == 0) && aligned16(X) && (ldx % 4 == 0) && aligned16(hi) &&
+                   aligned16(lo) && (ldh % 8 == 0);
+  const long long items = vec ? (long long)rows * (cols / 8) : (long long)rows * cols;
+  long long blocks = (items + 255) / 256;
+  const long long cap = (long long)h->sm_count * 16;
+  if (blocks > cap) blocks = cap;
+  if (blocks < 1) blocks = 1;
+  if (vec)
+    sgc::split_vec8_kernel<<<(unsigned)blocks, 256, 0, st>>>(rows, cols, X, ldx, hi, lo, ldh, s);
+  else
+    sgc::split_scalar_kernel<<<(unsigned)blocks, 256, 0, st>>>(rows, cols, X, ldx, hi, lo, ldh, s);
+  h->launches++;
+  return cudaGetLastError() == cudaSuccess ? SGEMM_CUBE_OK : SGEMM_CUBE_CUDA_ERROR;
+}
+
+// FP16-operand tensor-core GEMM launch, NTERMS = 1 (lo pointers unused) or 3.
+template <int NTERMS>
+int launch_tc_gemm(sgemm_cube_ctx* h, int M, int N, int K, const uint16_t* Ahi, const uint16_t* Alo,
+                   int64_t lda16, const uint16_t* Bhi, const uint16_t* Blo, int64_t ldb16, float* D,
+                   int64_t ldd, int accumulate, int order, int kblock, float inv_scale,
+                   cudaStream_t st) {
+  using Cfg = sgc::TcCfg<NTERMS>;
+  int rc = set_kernel_attrs(h);
+  if (rc) return rc;
+  CUtensorMap tmA0, tmA1, tmB0, tmB1;
+  const CUtensorMapSwizzle a_swz =
+      (Cfg::A_ROW_BYTES == 128) ? CU_TENSOR_MAP_SWIZZLE_128B : CU_TENSOR_MAP_SWIZZLE_64B;
+  rc = make_map(h, &tmA0, CU_TENSOR_MAP_DATA_TYPE_FLOAT16, 2, Ahi, K, M, lda16, Cfg::BK, sgc::kBM, a_swz);
+  if (rc) return rc;
+  rc = make_map(h, &tmB0, CU_TENSOR_MAP_DATA_TYPE_FLOAT16, 2, Bhi, N, K, ldb16, 64, Cfg::BK,
+                CU_TENSOR_MAP_SWIZZLE_128B);
+  if (rc) return rc;
+  if (NTERMS == 3) {
+    rc = make_map(h, &tmA1, CU_TENSOR_MAP_DATA_TYPE_FLOAT16, 2, Alo, K, M, lda16, Cfg::BK, sgc::kBM, a_swz);
+    if (rc) return rc;
+    rc = make_map(h, &tmB1, CU_TENSOR_MAP_DATA_TYPE_FLOAT16, 2, Blo, N, K, ldb16, 64, Cfg::BK,
+                  CU_TENSOR_MAP_SWIZZLE_128B);
+    if (rc) return rc;
+  } else {
+    tmA1 = tmA0;
+    tmB1 = tmB0;
+  }
+  sgc::TcGemmParams p;
+  p.M = M; p.N = N; p.K = K;
+  p.D = D; p.ldd = ldd;
+  p.accumulate = accumulate;
+  p.order = order;
+  p.kchunk_blocks = kblock / Cfg::BK;
+  if (p.kchunk_blocks < 1) p.kchunk_blocks = 1;
+  p.inv_scale = inv_scale;
+  p.err = h->err_dev;
+  p.A32 = nullptr; p.lda32 = 0; p.B32 = nullptr; p.ldb32 = 0; p.scale = 1.f;
+  const int tiles = ((M + sgc::kBM - 1) / sgc::kBM) * ((N + sgc::kBN - 1) / sgc::kBN);
+  const int grid = tiles < h->sm_count ? tiles : h->sm_count;
+  sgc::tc_gemm_kernel<NTERMS, false><<<grid, sgc::kTcThreads, Cfg::SMEM_BYTES, st>>>(tmA0, tmA1, tmB0, tmB1, p);
+  h->launches++;
+  return cudaGetLastError() == cudaSuccess ? SGEMM_CUBE_OK : SGEMM_CUBE_CUDA_ERROR;
+}
+
+int launch_fused(sgemm_cube_ctx* h, int M, int N, int K, const float* A, int64_t lda, const float* B,
+                 int64_t ldb, float* C, int64_t ldc, int s, int order, cudaStream_t st) {
+  using Cfg = sgc::TcCfg<3>;
+  int rc = set_kernel_attrs(h);
+  if (rc) return rc;
+  sgc::TcGemmParams p;
+  p.M = M; p.N = N; p.K = K;
+  p.D = C; p.ldd = ldc;
+  p.accumulate = 0;
+  p.order = order;
+  const int kblock = (order == SGEMM_CUBE_TERMWISE) ? h->kblock_termwise : h->kblock_elementwise;
+  p.kchunk_blocks = kblock / Cfg::BK;
+  if (p.kchunk_blocks < 1) p.kchunk_blocks = 1;
+  p.inv_scale = ldexpf(1.0f, -s);
+  p.err = h->err_dev;
+  p.A32 = A; p.lda32 = lda;
+  p.B32 = B; p.ldb32 = ldb;
+  p.scale = ldexpf(1.0f, s);
+  CUtensorMap unused;
+  memset(&unused, 0, sizeof(unused));
+  const int tiles = ((M + sgc::kBM - 1) / sgc::kBM) * ((N + sgc::kBN - 1) / sgc::kBN);
+  const int grid = tiles < h->sm_count ? tiles : h->sm_count;
+  sgc::tc_gemm_kernel<3, true><<<grid, sgc::kFusedThreads, Cfg::SMEM_BYTES, st>>>(unused, unused, unused, unused, p);
+  h->launches++;
+  return cudaGetLastError() == cudaSuccess ? SGEMM_CUBE_OK : SGEMM_CUBE_CUDA_ERROR;
+}
+
+}  // namespace
+
+extern "C" {
+
+int sgemm_cube_version(void) { return 100; }
+
+const char* sgemm_cube_status_string(int status) {
+  switch (status) {
+    case SGEMM_CUBE_OK: return "success";
+    case SGEMM_CUBE_INVALID_ARG: return "invalid argument";
+    case SGEMM_CUBE_MISALIGNED: return "pointer or leading dimension violates an alignment rule";
+    case SGEMM_CUBE_CUDA_ERROR: return "CUDA runtime or driver call failed";
+    case SGEMM_CUBE_DEVICE_TIMEOUT: return "a kernel gave up on a bounded wait";
+    case SGEMM_CUBE_UNSUPPORTED_ARCH: return "device is not compute capability 10.x (sm_100)";
+    case SGEMM_CUBE_ALLOC_FAILED: return "workspace allocation failed";
+    default: return "unknown status";
+  }
+}
+
+int sgemm_cube_create(sgemm_cube_handle* out, int device) {
+  if (!out) return SGEMM_CUBE_INVALID_ARG;
+  *out = nullptr;
+  int count = 0;
+  if (cudaGetDeviceCount(&count) != cudaSuccess) { cudaGetLastError(); return SGEMM_CUBE_CUDA_ERROR; }
+  if (device < 0 || device >= count) return SGEMM_CUBE_INVALID_ARG;
+  cudaDeviceProp prop;
+  if (cudaGetDeviceProperties(&prop, device) != cudaSuccess) return SGEMM_CUBE_CUDA_ERROR;
+  if (prop.major != 10) return SGEMM_CUBE_UNSUPPORTED_ARCH;
+  DeviceGuard g(device);
+  if (!g.ok) return SGEMM_CUBE_CUDA_ERROR;
+  sgemm_cube_ctx* h = new (std::nothrow) sgemm_cube_ctx();
+  if (!h) return SGEMM_CUBE_ALLOC_FAILED;
+  h->device = device;
+  h->sm_count = prop.multiProcessorCount;
+  void* fn = nullptr;
+  cudaDriverEntryPointQueryResult qres;
+  if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &qres) != cudaSuccess ||
+      qres != cudaDriverEntryPointSuccess || !fn) {
+    cudaGetLastError();
+    delete h;
+    return SGEMM_CUBE_CUDA_ERROR;
+  }
+  h->encode = reinterpret_cast<EncodeTiledFn>(fn);
+  if (cudaMalloc(reinterpret_cast<void**>(&h->err_dev), sizeof(unsigned int)) != cudaSuccess) {
+    cudaGetLastError();
+    delete h;
+    return SGEMM_CUBE_ALLOC_FAILED;
+  }
+  if (cudaMemset(h->err_dev, 0, sizeof(unsigned int)) != cudaSuccess) {
+    cudaFree(h->err_dev);
+    delete h;
+    return SGEMM_CUBE_CUDA_ERROR;
+  }
+  *out = h;
+  return SGEMM_CUBE_OK;
+}
+
+int sgemm_cube_destroy(sgemm_cube_handle h) {
+  if (!h) return SGEMM_CUBE_INVALID_ARG;
+  DeviceGuard g(h->device);
+  int rc = SGEMM_CUBE_OK;
+  if (cudaDeviceSynchronize() != cudaSuccess) rc = SGEMM_CUBE_CUDA_ERROR;
+  unsigned int e = 0;
+  if (rc == SGEMM_CUBE_OK && cudaMemcpy(&e, h->err_dev, sizeof(e), cudaMemcpyDeviceToHost) == cudaSuccess && e)
+    rc = SGEMM_CUBE_DEVICE_TIMEOUT;
+  if (h->ws) cudaFree(h->ws);
+  if (h->host_ws) cudaFree(h->host_ws);
+  cudaFree(h->err_dev);
+  delete h;
+  return rc;
+}
+
+int sgemm_cube_set_option(sgemm_cube_handle h, int option, int64_t value) {
+  if (!h) return SGEMM_CUBE_INVALID_ARG;
+  if (value < 64 || value % 64 != 0 || value > (1 << 24)) return SGEMM_CUBE_INVALID_ARG;
+  if (option == SGEMM_CUBE_OPT_TERMWISE_K_BLOCK) h->kblock_termwise = (int)value;
+  else if (option == SGEMM_CUBE_OPT_ELEMENTWISE_K_BLOCK) h->kblock_elementwise = (int)value;
+  else return SGEMM_CUBE_INVALID_ARG;
+  return SGEMM_CUBE_OK;
+}
+
+int sgemm_cube_split(sgemm_cube_handle h, int rows, int cols, const float* X, int64_t ldx,
+                     uint16_t* hi, uint16_t* lo, int64_t ldh, int scale_exp, void* stream) {
+  if (!h || !X || !hi || !lo) return SGEMM_CUBE_INVALID_ARG;
+  if (rows <= 0 || cols <= 0 || ldx < cols || ldh < cols) return SGEMM_CUBE_INVALID_ARG;
+  if (scale_exp < 0 || scale_exp > 24) return SGEMM_CUBE_INVALID_ARG;
+  DeviceGuard g(h->device);
+  if (!g.ok) return SGEMM_CUBE_CUDA_ERROR;
+  return launch_split(h, rows, cols, X, ldx, hi, lo, ldh, scale_exp, static_cast<cudaStream_t>(stream));
+}
+
+int sgemm_cube(sgemm_cube_handle h, int M, int N, int K, const float* A, int64_t lda, const float* B,
+               int64_t ldb, float* C, int64_t ldc, int scale_exp, int order, void* stream) {
+  if (!h || !A || !B || !C) return SGEMM_CUBE_INVALID_ARG;
+  int rc = check_gemm_dims(M, N, K, lda, ldb, ldc);
+  if (rc) return rc;
+  if (scale_exp < 0 || scale_exp > 24) return SGEMM_CUBE_INVALID_ARG;
+  if (order != SGEMM_CUBE_TERMWISE && order != SGEMM_CUBE_ELEMENTWISE) return SGEMM_CUBE_INVALID_ARG;
+  if (!aligned16(A) || !aligned16(B) || (lda % 4) || (ldb % 4)) return SGEMM_CUBE_MISALIGNED;
+  DeviceGuard g(h->device);
+  if (!g.ok) return SGEMM_CUBE_CUDA_ERROR;
+  return launch_fused(h, M, N, K, A, lda, B, ldb, C, ldc, scale_exp, order,
+                      static_cast<cudaStream_t>(stream));
+}
+
+int sgemm_cube_presplit(sgemm_cube_handle h, int M, int N, int K, const uint16_t* Ahi,
+                        const uint16_t* Alo, int64_t lda16, const uint16_t* Bhi, const uint16_t* Blo,
+                        int64_t ldb16, float* C, int64_t ldc, int scale_exp, int order, void* stream) {
+  if (!h || !Ahi || !Alo || !Bhi || !Blo || !C) return SGEMM_CUBE_INVALID_ARG;
+  int rc = check_gemm_dims(M, N, K, lda16, ldb16, ldc);
+  if (rc) return rc;
+  if (scale_exp < 0 || scale_exp > 24) return SGEMM_CUBE_INVALID_ARG;
+  if (order != SGEMM_CUBE_TERMWISE && order != SGEMM_CUBE_ELEMENTWISE) return SGEMM_CUBE_INVALID_ARG;
+  if (!aligned16(Ahi) || !aligned16(Alo) || !aligned16(Bhi) || !aligned16(Blo) || (lda16 % 8) ||
+      (ldb16 % 8))
+    return SGEMM_CUBE_MISALIGNED;
+  DeviceGuard g(h->device);
+  if (!g.ok) return SGEMM_CUBE_CUDA_ERROR;
+  const int kblock = (order == SGEMM_CUBE_TERMWISE) ? h->kblock_termwise : h->kblock_elementwise;
+  return launch_tc_gemm<3>(h, M, N, K, Ahi, Alo, lda16, Bhi, Blo, ldb16, C, ldc, 0, order, kblock,
+                           ldexpf(1.0f, -scale_exp), static_cast<cudaStream_t>(stream));
+}
+
+int sgemm_cube_hgemm(sgemm_cube_handle h, int M, int N, int K, const uint16_t* A16, int64_t lda16,
+                     const uint16_t* B16, int64_t ldb16, float* D, int64_t ldd, int accumulate,
+                     void* stream) {
+  if (!h || !A16 || !B16 || !D) return SGEMM_CUBE_INVALID_ARG;
+  int rc = check_gemm_dims(M, N, K, lda16, ldb16, ldd);
+  if (rc) return rc;
+  if (!aligned16(A16) || !aligned16(B16) || (lda16 % 8) || (ldb16 % 8)) return SGEMM_CUBE_MISALIGNED;
+  DeviceGuard g(h->device);
+  if (!g.ok) return SGEMM_CUBE_CUDA_ERROR;
+  return launch_tc_gemm<1>(h, M, N, K, A16, nullptr, lda16, B16, nullptr, ldb16, D, ldd,
+                           accumulate ? 1 : 0, 0, h->kblock_termwise, 1.0f,
+                           static_cast<cudaStream_t>(stream));
+}
+
+int sgemm_cube_unfused(sgemm_cube_handle h, int M, int N, int K, const float* A, int64_t lda,
+                       const float* B, int64_t ldb, float* C, int64_t ldc, int scale_exp, int order,
+                       void* stream) {
+  if (!h || !A || !B || !C) return SGEMM_CUBE_INVALID_ARG;
+  int rc = check_gemm_dims(M, N, K, lda, ldb, ldc);
+  if (rc) return rc;
+  if (scale_exp < 0 || scale_exp > 24) return SGEMM_CUBE_INVALID_ARG;
+  if (order != SGEMM_CUBE_TERMWISE) return SGEMM_CUBE_INVALID_ARG;
+  DeviceGuard g(h->device);
+  if (!g.ok) return SGEMM_CUBE_CUDA_ERROR;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  // Workspace layout: A_hi, A_lo (M x ldA16), B_hi, B_lo (K x ldB16), D_hh, D_x (M x ldD).
+  const size_t ldA16 = round_up((size_t)K, 8), ldB16 = round_up((size_t)N, 8);
+  const size_t ldD = round_up((size_t)N, 4);
+  const size_t szA = round_up((size_t)M * ldA16 * 2, 256), szB = round_up((size_t)K * ldB16 * 2, 256);
+  const size_t szD = round_up((size_t)M * ldD * 4, 256);
+  rc = grow(&h->ws, &h->ws_bytes, 2 * szA + 2 * szB + 2 * szD);
+  if (rc) return rc;
+  uint8_t* w = static_cast<uint8_t*>(h->ws);
+  uint16_t* Ahi = reinterpret_cast<uint16_t*>(w);
+  uint16_t* Alo = reinterpret_cast<uint16_t*>(w + szA);
+  uint16_t* Bhi = reinterpret_cast<uint16_t*>(w + 2 * szA);
+  uint16_t* Blo = reinterpret_cast<uint16_t*>(w + 2 * szA + szB);
+  float* Dhh = reinterpret_cast<float*>(w + 2 * szA + 2 * szB);
+  float* Dx = reinterpret_cast<float*>(w + 2 * szA + 2 * szB + szD);
+  const float inv = ldexpf(1.0f, -scale_exp);
+  const int kb = h->kblock_termwise;
+  if ((rc = launch_split(h, M, K, A, lda, Ahi, Alo, (int64_t)ldA16, scale_exp, st))) return rc;
+  if ((rc = launch_split(h, K, N, B, ldb, Bhi, Blo, (int64_t)ldB16, scale_exp, st))) return rc;
+  if ((rc = launch_tc_gemm<1>(h, M, N, K, Ahi, nullptr, ldA16, Bhi, nullptr, ldB16, Dhh, ldD, 0, 0, kb, 1.f, st))) return rc;
+  if ((rc = launch_tc_gemm<1>(h, M, N, K, Alo, nullptr, ldA16, Bhi, nullptr, ldB16, Dx, ldD, 0, 0, kb, 1.f, st))) return rc;
+  if ((rc = launch_tc_gemm<1>(h, M, N, K, Ahi, nullptr, ldA16, Blo, nullptr, ldB16, Dx, ldD, 1, 0, kb, 1.f, st))) return rc;
+  const long long total = (long long)M * N;
+  long long blocks = (total + 255) / 256;
+  const long long cap = (long long)h->sm_count * 16;
+  if (blocks > cap) blocks = cap;
+  sgc::combine_kernel<<<(unsigned)blocks, 256, 0, st>>>(M, N, Dhh, Dx, (long long)ldD, C, ldc, inv);
+  h->launches++;
+  return cudaGetLastError() == cudaSuccess ? SGEMM_CUBE_OK : SGEMM_CUBE_CUDA_ERROR;
+}
+
+int sgemm_cube_host(sgemm_cube_handle h, int M, int N, int K, const float* A_host, int64_t lda,
+                    const float* B_host, int64_t ldb, float* C_host, int64_t ldc, int scale_exp,
+                    int order, void* stream) {
+  if (!h || !A_host || !B_host || !C_host) return SGEMM_CUBE_INVALID_ARG;
+  int rc = check_gemm_dims(M, N, K, lda, ldb, ldc);
+  if (rc) return rc;
+  if (scale_exp < 0 || scale_exp > 24) return SGEMM_CUBE_INVALID_ARG;
+  if (order != SGEMM_CUBE_TERMWISE && order != SGEMM_CUBE_ELEMENTWISE) return SGEMM_CUBE_INVALID_ARG;
+  DeviceGuard g(h->device);
+  if (!g.ok) return SGEMM_CUBE_CUDA_ERROR;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  const size_t ldA = round_up((size_t)K, 4), ldB = round_up((size_t)N, 4), ldC = ldB;
+  const size_t szA = round_up((size_t)M * ldA * 4, 256), szB = round_up((size_t)K * ldB * 4, 256);
+  const size_t szC = round_up((size_t)M * ldC * 4, 256);
+  rc = grow(&h->host_ws, &h->host_ws_bytes, szA + szB + szC);
+  if (rc) return rc;
+  uint8_t* w = static_cast<uint8_t*>(h->host_ws);
+  float* dA = reinterpret_cast<float*>(w);
+  float* dB = reinterpret_cast<float*>(w + szA);
+  float* dC = reinterpret_cast<float*>(w + szA + szB);
+  if (cudaMemcpy2DAsync(dA, ldA * 4, A_host, (size_t)lda * 4, (size_t)K * 4, M, cudaMemcpyHostToDevice, st) != cudaSuccess ||
+      cudaMemcpy2DAsync(dB, ldB * 4, B_host, (size_t)ldb * 4, (size_t)N * 4, K, cudaMemcpyHostToDevice, st) != cudaSuccess) {
+    cudaGetLastError();
+    return SGEMM_CUBE_CUDA_ERROR;
+  }
+  rc = launch_fused(h, M, N, K, dA, (int64_t)ldA, dB, (int64_t)ldB, dC, (int64_t)ldC, scale_exp, order, st);
+  if (rc) return rc;
+  if (cudaMemcpy2DAsync(C_host, (size_t)ldc * 4, dC, ldC * 4, (size_t)N * 4, M, cudaMemcpyDeviceToHost, st) != cudaSuccess) {
+    cudaGetLastError();
+    return SGEMM_CUBE_CUDA_ERROR;
+  }
+  return sgemm_cube_check(h, stream, nullptr);
+}
+
+int sgemm_cube_check(sgemm_cube_handle h, void* stream, uint32_t* detail_out) {
+  if (!h) return SGEMM_CUBE_INVALID_ARG;
+  DeviceGuard g(h->device);
+  if (!g.ok) return SGEMM_CUBE_CUDA_ERROR;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  if (cudaStreamSynchronize(st) != cudaSuccess) { cudaGetLastError(); return SGEMM_CUBE_CUDA_ERROR; }
+  unsigned int e = 0;
+  if (cudaMemcpy(&e, h->err_dev, sizeof(e), cudaMemcpyDeviceToHost) != cudaSuccess) {
+    cudaGetLastError();
+    return SGEMM_CUBE_CUDA_ERROR;
+  }
+  if (detail_out) *detail_out = e;
+  if (e) {
+    cudaMemset(h->err_dev, 0, sizeof(e));
+    return SGEMM_CUBE_DEVICE_TIMEOUT;
+  }
+  return SGEMM_CUBE_OK;
+}
+
+int64_t sgemm_cube_launch_count(sgemm_cube_handle h) { return h ? h->launches : -1; }
+
+}  // extern "C"

@@ -100,3 +100,12 @@ def make_pair(kind: str, seed: int, M: int, N: int, K: int):
     if kind == "normal":
         return normal(seed, (M, K), 0), normal(seed, (K, N), 1)
     raise ValueError("unknown workload kind: %r" % (kind,))
+
+
+def device_normal(seed: int, shape, device="cuda:0"):
+    """i.i.d. N(0, 1) FP32 generated on the device with a seeded torch generator, for the
+    full-size workloads where host generation would dominate the run."""
+    import torch
+    g = torch.Generator(device=device)
+    g.manual_seed(int(seed))
+    return torch.randn(tuple(shape), generator=g, device=device, dtype=torch.float32)

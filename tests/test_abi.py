@@ -1,0 +1,67 @@
+"""CPU-side checks of the boundary: the CUDA library builds for sm_100a, loads, and exports every
+symbol that include/sgemm_cube.h declares.  No compute call is made here."""
+import ctypes
+import os
+import re
+
+import pytest
+
+from paper_2507_23387_b200 import binding, build
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+@pytest.fixture(scope="module")
+def lib():
+    build.build()
+    return ctypes.CDLL(build.LIB)
+
+
+def _declared_functions():
+    text = open(os.path.join(ROOT, "include", "sgemm_cube.h")).read()
+    text = re.sub(r"/\*.*?\*/", "", text, flags=re.S)
+    names = re.findall(r"\b(sgemm_cube\w*)\s*\(", text)
+    return sorted(set(names))
+
+
+def test_header_declares_the_documented_entry_points():
+    names = _declared_functions()
+    for must in ("sgemm_cube_create", "sgemm_cube_destroy", "sgemm_cube_split", "sgemm_cube",
+                 "sgemm_cube_unfused"):
+        assert must in names
+
+
+def test_library_exports_every_declared_symbol(lib):
+    for name in _declared_functions():
+        assert hasattr(lib, name), "missing export: %s" % name
+
+
+def test_binding_lists_every_declared_symbol():
+    assert sorted(binding.EXPORTS) == _declared_functions()
+
+
+def test_status_strings_and_version(lib):
+    lib.sgemm_cube_status_string.restype = ctypes.c_char_p
+    seen = set()
+    for code in range(7):
+        s = lib.sgemm_cube_status_string(code)
+        assert s and s not in seen
+        seen.add(s)
+    assert lib.sgemm_cube_status_string(99) == b"unknown status"
+    assert lib.sgemm_cube_version() >= 100
+
+
+def test_null_arguments_are_rejected_without_a_device(lib):
+    lib.sgemm_cube_create.argtypes = [ctypes.c_void_p, ctypes.c_int]
+    assert lib.sgemm_cube_create(None, 0) == binding.INVALID_ARG
+    lib.sgemm_cube_destroy.argtypes = [ctypes.c_void_p]
+    assert lib.sgemm_cube_destroy(None) == binding.INVALID_ARG
+    lib.sgemm_cube_check.argtypes = [ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p]
+    assert lib.sgemm_cube_check(None, None, None) == binding.INVALID_ARG
+
+
+def test_binding_fails_loudly_when_library_is_missing(monkeypatch, tmp_path):
+    monkeypatch.setattr(binding, "_lib", None)
+    monkeypatch.setattr(binding, "LIB_PATH", str(tmp_path / "nope.so"))
+    with pytest.raises(OSError):
+        binding.load()

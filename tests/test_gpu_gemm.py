@@ -1,0 +1,290 @@
+"""GPU parity of the SGEMM-cube GEMM entry points against the oracle.
+
+Bit-exact where the arithmetic is exact (inputs whose partial sums need no rounding); elsewhere
+the three gates of gpu_common.gates: componentwise 2 K 2^-24 (|A||B|) against FP64, and at most
+twice the oracle's own componentwise and Frobenius error.  Full-size configurations are checked
+on sampled rows, which the oracle computes one by one.
+"""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from paper_2507_23387_b200 import binding, inputs
+from gpu_common import K_BLOCK, gates, padded_dev, to_dev
+
+pytestmark = pytest.mark.gpu
+
+T, E = binding.TERMWISE, binding.ELEMENTWISE
+
+
+@pytest.fixture(scope="module")
+def handle():
+    h = binding.Handle(0)
+    yield h
+    st, det = h.sgemm_cube_check()
+    h.destroy()
+    assert st == 0, hex(det)
+
+
+def run(h, path, Ad, Bd, s, order):
+    """Run one entry point on device operands; returns C as numpy."""
+    M, N = Ad.shape[0], Bd.shape[1]
+    C = torch.full((M, N), float("nan"), device="cuda:0")
+    if path == "fused":
+        h.sgemm_cube(Ad, Bd, C, s, order)
+    elif path == "unfused":
+        h.sgemm_cube_unfused(Ad, Bd, C, s, order)
+    elif path == "presplit":
+        K = Ad.shape[1]
+        K8, N8 = (K + 7) // 8 * 8, (N + 7) // 8 * 8
+        f16 = dict(dtype=torch.float16, device="cuda:0")
+        Ahi, Alo = torch.empty((M, K8), **f16)[:, :K], torch.empty((M, K8), **f16)[:, :K]
+        Bhi, Blo = torch.empty((K, N8), **f16)[:, :N], torch.empty((K, N8), **f16)[:, :N]
+        h.sgemm_cube_split(Ad, Ahi, Alo, s)
+        h.sgemm_cube_split(Bd, Bhi, Blo, s)
+        h.sgemm_cube_presplit(Ahi, Alo, Bhi, Blo, C, s, order)
+    st, det = h.sgemm_cube_check()
+    assert st == 0, "device error %s" % hex(det)
+    return C.cpu().numpy()
+
+
+PATHS = [("fused", T), ("fused", E), ("presplit", T), ("presplit", E), ("unfused", T)]
+
+
+@pytest.mark.parametrize("path,order", PATHS)
+def test_small_integers_exact(handle, path, order):
+    rng = np.random.default_rng(1)
+    for (M, N, K) in [(5, 7, 11), (128, 256, 64), (130, 260, 100), (300, 520, 72)]:
+        A = rng.integers(-8, 9, size=(M, K)).astype(np.float32)
+        B = rng.integers(-8, 9, size=(K, N)).astype(np.float32)
+        C = run(handle, path, padded_dev(A, 4), padded_dev(B, 4), 11, order)
+        want = (A.astype(np.int64) @ B.astype(np.int64)).astype(np.float32)
+        assert np.array_equal(C, want), (M, N, K)
+        assert np.array_equal(C, oracle.sgemm_cube(A, B, 11, order, K_BLOCK[order]))
+
+
+@pytest.mark.parametrize("path,order", PATHS)
+@pytest.mark.parametrize("s", [9, 11, 12])
+def test_three_terms_kept_low_low_dropped_bit_exact(handle, path, order, s):
+    # x = p + q 2^-13 (p in 4..7, q in -3..3): every partial sum of the three computed products is
+    # exact in FP32, whatever the summation order or rounding mode, so the CUDA result must equal
+    # the oracle's bit for bit, and both must equal the closed form without the q q' 2^-26 term.
+    rng = np.random.default_rng(2)
+    M, N, K = 200, 264, 48
+    pA, qA = rng.integers(4, 8, (M, K)), rng.integers(-3, 4, (M, K))
+    pB, qB = rng.integers(4, 8, (K, N)), rng.integers(-3, 4, (K, N))
+    sgA, sgB = rng.choice([-1, 1], (M, K)), rng.choice([-1, 1], (K, N))
+    A = (sgA * (pA + qA * 2.0 ** -13)).astype(np.float32)
+    B = (sgB * (pB + qB * 2.0 ** -13)).astype(np.float32)
+    want = ((sgA * pA) @ (sgB * pB)
+            + ((sgA * pA) @ (sgB * qB) + (sgA * qA) @ (sgB * pB)) * 2.0 ** -13)
+    C = run(handle, path, to_dev(A), to_dev(B), s, order)
+    assert np.array_equal(C.astype(np.float64), want)
+    assert np.array_equal(C, oracle.sgemm_cube(A, B, s, order, K_BLOCK[order]))
+
+
+@pytest.mark.parametrize("path,order", PATHS)
+@pytest.mark.parametrize("seed", [0, 1, 2, 3, 4])
+def test_config1_256_cubed_uniform(handle, path, order, seed):
+    A, B = inputs.make_pair("uniform_pm1", seed, 256, 256, 256)
+    C = run(handle, path, to_dev(A), to_dev(B), 11, order)
+    gates(C, A, B, 11, order, label="%s order %d seed %d" % (path, order, seed))
+
+
+@pytest.mark.parametrize("path,order", PATHS)
+@pytest.mark.parametrize("shape", [(1, 1, 1), (129, 257, 33), (200, 300, 136), (384, 768, 1000),
+                                   (127, 8, 2049), (640, 1280, 96)])
+def test_ragged_shapes(handle, path, order, shape):
+    M, N, K = shape
+    A, B = inputs.make_pair("normal", 11, M, N, K)
+    C = run(handle, path, padded_dev(A, 4), padded_dev(B, 4), 11, order)
+    gates(C, A, B, 11, order, label="%s %s" % (path, shape))
+
+
+@pytest.mark.parametrize("path,order", [("fused", T), ("fused", E), ("presplit", T)])
+def test_output_leading_dimension_and_alignment(handle, path, order):
+    M, N, K = 150, 203, 77
+    A, B = inputs.make_pair("normal", 5, M, N, K)
+    Ad, Bd = padded_dev(A, 4), padded_dev(B, 4)
+    big = torch.full((M, 211), -7.0, device="cuda:0")
+    Cv = big[:, 3:3 + N]                       # ldc = 211, pointer offset 12 bytes: scalar stores
+    if path == "fused":
+        handle.sgemm_cube(Ad, Bd, Cv, 11, order)
+    else:
+        Ahi, Alo = (torch.empty((M, 80), dtype=torch.float16, device="cuda:0")[:, :K] for _ in range(2))
+        Bhi, Blo = (torch.empty((K, 208), dtype=torch.float16, device="cuda:0")[:, :N] for _ in range(2))
+        handle.sgemm_cube_split(Ad, Ahi, Alo, 11)
+        handle.sgemm_cube_split(Bd, Bhi, Blo, 11)
+        handle.sgemm_cube_presplit(Ahi, Alo, Bhi, Blo, Cv, 11, order)
+    assert handle.sgemm_cube_check()[0] == 0
+    gates(Cv.cpu().numpy(), A, B, 11, order)
+    assert torch.all(big[:, :3] == -7.0) and torch.all(big[:, 3 + N:] == -7.0)
+
+
+def test_fused_and_presplit_agree_bitwise(handle):
+    # Same products, same accumulation structure: the on-the-fly split must reproduce the words of
+    # the split kernel exactly, so the two results are identical.
+    A, B = inputs.make_pair("exponent_spread", 4, 384, 512, 640)
+    for order in (T, E):
+        C1 = run(handle, "fused", to_dev(A), to_dev(B), 11, order)
+        C2 = run(handle, "presplit", to_dev(A), to_dev(B), 11, order)
+        assert np.array_equal(C1, C2)
+
+
+def test_k_block_option_changes_bracketing_not_validity(handle):
+    A, B = inputs.make_pair("uniform_pm1", 3, 256, 256, 2048)
+    Ad, Bd = to_dev(A), to_dev(B)
+    try:
+        for kb in (64, 128, 512):
+            handle.sgemm_cube_set_option(binding.OPT_TERMWISE_K_BLOCK, kb)
+            C = run(handle, "fused", Ad, Bd, 11, T)
+            gates(C, A, B, 11, T, kb=kb, label="kblock %d" % kb)
+    finally:
+        handle.sgemm_cube_set_option(binding.OPT_TERMWISE_K_BLOCK, K_BLOCK[T])
+    with pytest.raises(binding.SgemmCubeError):
+        handle.sgemm_cube_set_option(binding.OPT_TERMWISE_K_BLOCK, 100)
+
+
+def _sampled_rows_check(handle, path, order, A_rows_np, B_np, C_dev, rows, label):
+    C_rows = C_dev[torch.as_tensor(rows, device="cuda:0")].cpu().numpy()
+    return gates(C_rows, A_rows_np, B_np, 11, order, label=label)
+
+
+@pytest.mark.parametrize("path,order", PATHS)
+def test_config2_4096_cubed_sampled_rows(handle, path, order):
+    n = 4096
+    A, B = inputs.make_pair("uniform_pm1", 0, n, n, n)
+    rows = np.sort(np.random.default_rng(0).choice(n, 48, replace=False))
+    Ad, Bd = to_dev(A), to_dev(B)
+    C = torch.empty((n, n), device="cuda:0")
+    getattr(handle, "sgemm_cube" if path == "fused" else "sgemm_cube_unfused")(Ad, Bd, C, 11, order) \
+        if path != "presplit" else None
+    if path == "presplit":
+        C = torch.from_numpy(run(handle, path, Ad, Bd, 11, order)).to("cuda:0")
+    assert handle.sgemm_cube_check()[0] == 0
+    _sampled_rows_check(handle, path, order, A[rows], B, C, rows, "4096^3 %s %d" % (path, order))
+
+
+def test_config2_orders_compared(handle):
+    # Both orders run on the same 4096^3 input; each passes its gates (above); here their errors
+    # are put side by side on sampled rows, as the configuration asks.
+    n = 4096
+    A, B = inputs.make_pair("uniform_pm1", 1, n, n, n)
+    rows = np.arange(0, n, 128)
+    Ad, Bd = to_dev(A), to_dev(B)
+    C64, AB = oracle.dgemm_ref(A[rows], B)
+    errs = {}
+    for order in (T, E):
+        C = torch.empty((n, n), device="cuda:0")
+        handle.sgemm_cube(Ad, Bd, C, 11, order)
+        assert handle.sgemm_cube_check()[0] == 0
+        errs[order] = oracle.frobenius_rel_err(C[torch.as_tensor(rows, device="cuda:0")].cpu().numpy(), C64)
+    assert errs[T] < 2e-6 and errs[E] < 2e-6
+    assert 0.25 < errs[T] / errs[E] < 4.0
+
+
+@pytest.mark.parametrize("path,order", [("fused", T), ("presplit", T), ("unfused", T)])
+def test_config3_8192_cubed_exponent_spread_sampled_rows(handle, path, order):
+    n = 8192
+    A, B = inputs.make_pair("exponent_spread", 0, n, n, n)
+    rows = np.sort(np.random.default_rng(1).choice(n, 24, replace=False))
+    Ad, Bd = to_dev(A), to_dev(B)
+    C = torch.from_numpy(run(handle, path, Ad, Bd, 11, order))
+    gates(C[torch.as_tensor(rows)].numpy(), A[rows], B, 11, order, label="8192^3 %s" % path)
+
+
+@pytest.mark.parametrize("path,order", [("fused", T), ("fused", E), ("presplit", T), ("unfused", T)])
+def test_config4_long_k_normal(handle, path, order):
+    M = N = 1024
+    K = 65536
+    A, B = inputs.make_pair("normal", 0, M, N, K)
+    rows = np.arange(0, M, 32)
+    C = run(handle, path, to_dev(A), to_dev(B), 11, order)
+    gates(C[rows], A[rows], B, 11, order, label="long-K %s %d" % (path, order))
+
+
+def test_config4_error_growth_termwise_vs_elementwise(handle):
+    # Error as K grows (N(0,1) inputs): both orders stay far below the plain FP32 sequential sum
+    # at long K, and neither grows faster than sqrt(K) x 4.
+    M = N = 256
+    res = {}
+    for K in (1024, 16384, 65536):
+        A, B = inputs.make_pair("normal", 2, M, N, K)
+        C64 = oracle.dgemm_ref(A, B, with_abs=False)
+        for order in (T, E):
+            res[(K, order)] = oracle.frobenius_rel_err(run(handle, "fused", to_dev(A), to_dev(B), 11, order), C64)
+        res[(K, "f32")] = oracle.frobenius_rel_err(oracle.sgemm_f32(A, B), C64)
+    for order in (T, E):
+        assert res[(65536, order)] < res[(65536, "f32")] / 2
+        assert res[(65536, order)] < 4 * 8 * res[(1024, order)]
+
+
+@pytest.mark.parametrize("shape", [(16384, 16384, 1024), (12288, 12288, 12288)])
+def test_config5_large_shapes_sampled_rows(handle, shape):
+    M, N, K = shape
+    A = inputs.device_normal(0, (M, K))
+    B = inputs.device_normal(1, (K, N))
+    C = torch.empty((M, N), device="cuda:0")
+    handle.sgemm_cube(A, B, C, 11, T)
+    assert handle.sgemm_cube_check()[0] == 0
+    rows = np.sort(np.random.default_rng(2).choice(M, 8, replace=False))
+    idx = torch.as_tensor(rows, device="cuda:0")
+    gates(C[idx].cpu().numpy(), A[idx].cpu().numpy(), B.cpu().numpy(), 11, T, label=str(shape))
+    # properties that hold at any size: a permutation of A's rows permutes C's rows exactly
+    perm = torch.randperm(256, device="cuda:0", generator=torch.Generator("cuda:0").manual_seed(0))
+    A2 = A[:256][perm].contiguous()
+    C2 = torch.empty((256, N), device="cuda:0")
+    handle.sgemm_cube(A2, B, C2, 11, T)
+    assert torch.equal(C2, C[:256][perm])
+
+
+def test_hgemm_matches_fp64_product_of_fp16_inputs(handle):
+    for (M, N, K) in [(128, 256, 64), (200, 300, 136), (1024, 1024, 1024)]:
+        A = inputs.normal(1, (M, (K + 7) // 8 * 8))[:, :K]
+        B = inputs.normal(2, (K, (N + 7) // 8 * 8))[:, :N]
+        Ad = padded_dev(A.astype(np.float16), 8)
+        Bd = padded_dev(B.astype(np.float16), 8)
+        D = torch.full((M, N), float("nan"), device="cuda:0")
+        handle.sgemm_cube_hgemm(Ad, Bd, D)
+        ref = A.astype(np.float16).astype(np.float64) @ B.astype(np.float16).astype(np.float64)
+        AB = np.abs(A.astype(np.float16).astype(np.float64)) @ np.abs(B.astype(np.float16).astype(np.float64))
+        assert np.all(np.abs(D.cpu().numpy() - ref) <= 2 * K * 2.0 ** -24 * AB)
+        D2 = D.clone()
+        handle.sgemm_cube_hgemm(Ad, Bd, D2, accumulate=True)
+        assert np.allclose(D2.cpu().numpy(), 2 * D.cpu().numpy(), rtol=0, atol=0)
+
+
+def test_argument_errors(handle):
+    A = torch.zeros((8, 16), device="cuda:0")
+    B = torch.zeros((16, 8), device="cuda:0")
+    C = torch.zeros((8, 8), device="cuda:0")
+    lib = binding.load()
+    p = lambda t: t.data_ptr()
+    call = lambda **kw: lib.sgemm_cube(handle._h, kw.get("M", 8), kw.get("N", 8), kw.get("K", 16),
+                                       kw.get("A", p(A)), kw.get("lda", 16), kw.get("B", p(B)),
+                                       kw.get("ldb", 8), kw.get("C", p(C)), kw.get("ldc", 8),
+                                       kw.get("s", 11), kw.get("order", 0), None)
+    assert call() == binding.OK
+    assert call(M=0) == binding.INVALID_ARG
+    assert call(K=-1) == binding.INVALID_ARG
+    assert call(lda=15) == binding.INVALID_ARG
+    assert call(ldc=7) == binding.INVALID_ARG
+    assert call(s=25) == binding.INVALID_ARG
+    assert call(order=2) == binding.INVALID_ARG
+    assert call(A=None) == binding.INVALID_ARG
+    assert call(A=p(A) + 4) == binding.MISALIGNED
+    assert call(lda=18) == binding.MISALIGNED
+    assert lib.sgemm_cube_unfused(handle._h, 8, 8, 16, p(A), 16, p(B), 8, p(C), 8, 11, 1,
+                                  None) == binding.INVALID_ARG       # unfused is termwise only
+    assert handle.sgemm_cube_check()[0] == 0
+
+
+def test_host_buffer_entry_point(handle):
+    M, N, K = 300, 520, 200
+    A, B = inputs.make_pair("normal", 8, M, N, K)
+    Ah, Bh = torch.from_numpy(A).pin_memory(), torch.from_numpy(B).pin_memory()
+    Ch = torch.empty((M, N)).pin_memory()
+    handle.sgemm_cube_host(Ah, Bh, Ch, 11, T)
+    Cd = run(handle, "fused", padded_dev(A, 4), padded_dev(B, 4), 11, T)
+    assert np.array_equal(Ch.numpy(), Cd)

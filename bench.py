@@ -1,0 +1,327 @@
+#!/usr/bin/env python
+"""Benchmark of the SGEMM-cube hot path on B200.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference]
+
+One "step" is one pass of the whole hot path over one batch of synthetic input: a single call of
+the fused `sgemm_cube` entry point (operand split, three FP16 tensor-core products and the FP32
+reconstruction in one kernel) on M = N = K = 8192 FP32 matrices whose entries are
+(+/-) u * 2^e, u uniform in [1, 2), e a uniform integer in [-10, 10], with s = 11 and termwise
+accumulation.  The metric is FP32-equivalent TFLOP/s = 2 M N K / t.
+
+Prints ONE JSON line (rank 0).  `value` is measured with the operands resident in device memory;
+`e2e` through the host-buffer entry point with both copies inside the timed region; `roofline`
+compares the kernel's 3 x 2MNK FP16 tensor-core FLOPs per launch with the measured dense
+tensor-core peak; `cpu_baseline` is the CPU oracle timed on a bounded sample of the same
+workload.  With --impl reference the oracle itself is the timed arm.
+"""
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import threading
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+sys.path.insert(0, ROOT)
+
+M = N = K = 8192
+SCALE_EXP = 11
+WORKLOAD = "M=N=K=8192 FP32 GEMM, entries (+/-)u*2^e, u~U[1,2), e~U{-10..10}, s=11, termwise"
+METRIC = "FP32-equiv TFLOP/s (2MNK/t) at 8192^3"
+UNIT = "TFLOP/s"
+
+# DRAM traffic of one launch of the fused kernel at this workload, from the ncu capture summarised
+# in profiles/ (dram__bytes_read.sum + dram__bytes_write.sum); None until a capture exists.
+FUSED_KERNEL_DRAM_BYTES_PER_LAUNCH = None
+
+
+def measured_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as f:
+            d = json.load(f)
+        return {"bf16_tflops": float(d["bf16_tflops"]),
+                "bf16_tflops_sustained": float(d.get("bf16_tflops_sustained", d["bf16_tflops"])),
+                "hbm_gbs": float(d["hbm_gbs"]), "source": "measured"}
+    return {"bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0, "hbm_gbs": 6650.0,
+            "source": "fallback"}
+
+
+class ClockSampler:
+    """Samples nvidia-smi clocks and throttle reasons while the timed region runs."""
+    FIELDS = ("clocks.sm,clocks.max.sm,clocks_event_reasons.hw_slowdown,"
+              "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+              "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, gpu_index):
+        self.gpu = gpu_index
+        self.samples = []
+        self.proc = None
+        self.thread = None
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", "-i", str(self.gpu), "--query-gpu=" + self.FIELDS,
+                 "--format=csv,noheader,nounits", "-lms", "20"],
+                stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+        except OSError:
+            self.proc = None
+            return
+        self.thread = threading.Thread(target=self._read, daemon=True)
+        self.thread.start()
+
+    def _read(self):
+        for line in self.proc.stdout:
+            parts = [p.strip() for p in line.split(",")]
+            if len(parts) >= 6:
+                self.samples.append(parts)
+
+    def stop(self):
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except subprocess.TimeoutExpired:
+            self.proc.kill()
+        sm, mx, reasons = [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for s in self.samples:
+            try:
+                sm.append(float(s[0]))
+                mx.append(float(s[1]))
+            except ValueError:
+                continue
+            for name, v in zip(names, s[2:6]):
+                if v.lower().startswith("active"):
+                    reasons.add(name)
+        return {"sm_mhz": statistics.median(sm) if sm else None,
+                "sm_max_mhz": max(mx) if mx else None, "reasons": sorted(reasons),
+                "samples": len(sm)}
+
+
+def cpu_oracle_sample(rows):
+    """Time the oracle (as it stands) on `rows` rows of the workload; returns (TFLOP/s, s, threads)."""
+    import oracle
+    from paper_2507_23387_b200 import inputs
+    A = inputs.exponent_spread(0, (rows, K), stream=0)
+    B = inputs.exponent_spread(0, (K, N), stream=1)
+    oracle.sgemm_cube(A[:1], B[:, :8].copy(), SCALE_EXP, oracle.TERMWISE, 64)      # load the library
+    t0 = time.perf_counter()
+    oracle.sgemm_cube(A, B, SCALE_EXP, oracle.TERMWISE, 64)
+    dt = time.perf_counter() - t0
+    return 2.0 * rows * N * K / dt / 1e12, dt, oracle.num_threads()
+
+
+def run_reference(args, rank):
+    """The reference arm: the CPU oracle, timed on a bounded sample per step."""
+    if rank != 0:
+        return
+    import oracle
+    from paper_2507_23387_b200 import inputs
+    rows = 128
+    A = inputs.exponent_spread(0, (rows, K), stream=0)
+    B = inputs.exponent_spread(0, (K, N), stream=1)
+    for _ in range(max(1, min(args.warmup, 1))):
+        oracle.sgemm_cube(A[:8], B, SCALE_EXP, oracle.TERMWISE, 64)
+    steps = max(1, min(args.steps, 5))
+    t0 = time.perf_counter()
+    for _ in range(steps):
+        oracle.sgemm_cube(A, B, SCALE_EXP, oracle.TERMWISE, 64)
+    dt = (time.perf_counter() - t0) / steps
+    val = 2.0 * rows * N * K / dt / 1e12
+    sample = "%d of %d rows of A against the full B (split of B included), per step" % (rows, M)
+    print(json.dumps({
+        "impl": "reference", "metric": METRIC, "value": val, "unit": UNIT, "n_gpus": args.gpus,
+        "steps": steps, "warmup": args.warmup, "ms_per_step": dt * 1e3, "higher_is_better": True,
+        "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
+        "config": {"workload": WORKLOAD, "sample": sample},
+        "cpu_baseline": {"value": val, "unit": UNIT, "cores": oracle.num_threads(), "kind": "oracle",
+                         "sample": sample},
+        "e2e": {"value": val, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0}))
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--e2e-steps", type=int, default=3)
+    ap.add_argument("--cpu-rows", type=int, default=2048)
+    ap.add_argument("--size", type=int, default=8192,
+                    help="M = N = K; values other than 8192 are for profiler captures only")
+    ap.add_argument("--kernel-only", action="store_true",
+                    help="skip the ablation, end-to-end and CPU legs (profiler captures)")
+    args = ap.parse_args()
+    global M, N, K, WORKLOAD
+    if args.size != 8192:
+        M = N = K = args.size
+        WORKLOAD = WORKLOAD.replace("8192", str(args.size)) + " (reduced size: not a bench value)"
+
+    rank = int(os.environ.get("RANK", "0"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+
+    if args.impl == "reference":
+        run_reference(args, rank)
+        return
+
+    import torch
+    import torch.distributed as dist
+    from paper_2507_23387_b200 import binding, inputs
+
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the library has no CPU fallback")
+    torch.cuda.set_device(local_rank)
+    dev = "cuda:%d" % local_rank
+    if world > 1:
+        os.environ.setdefault("MASTER_ADDR", "127.0.0.1")
+        dist.init_process_group("nccl", device_id=torch.device(dev))
+
+    h = binding.Handle(local_rank)
+    # Same seeded workload on every rank (independent replicas of the problem: weak scaling).
+    A_host = torch.from_numpy(inputs.exponent_spread(0, (M, K), stream=0))
+    B_host = torch.from_numpy(inputs.exponent_spread(0, (K, N), stream=1))
+    A, B = A_host.to(dev), B_host.to(dev)
+    C = torch.empty((M, N), device=dev)
+    warmup = max(3, args.warmup)
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    for _ in range(warmup):
+        h.sgemm_cube(A, B, C, SCALE_EXP, binding.TERMWISE)
+    barrier()
+    sampler = ClockSampler(local_rank)
+    sampler.start()
+    launches0 = h.sgemm_cube_launch_count()
+    ev = [torch.cuda.Event(enable_timing=True) for _ in range(args.steps + 1)]
+    barrier()
+    ev[0].record()
+    for i in range(args.steps):
+        h.sgemm_cube(A, B, C, SCALE_EXP, binding.TERMWISE)
+        ev[i + 1].record()
+    barrier()
+    total_ms = ev[0].elapsed_time(ev[-1])
+    clocks = sampler.stop()
+    launches = h.sgemm_cube_launch_count() - launches0
+    st, det = h.sgemm_cube_check()
+    if st != 0:
+        raise SystemExit("device error %s" % hex(det))
+    per_launch_ms = [ev[i].elapsed_time(ev[i + 1]) for i in range(args.steps)]
+    t = torch.tensor([total_ms], device=dev, dtype=torch.float64)
+    if world > 1:
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    total_ms = float(t.item())
+    ms_per_step = total_ms / args.steps
+    flops = 2.0 * M * N * K
+    value = world * flops / (ms_per_step * 1e-3) / 1e12
+
+    # Ablation legs on rank 0 (not part of `value`): pre-split kernel, unfused path, split alone.
+    extra = {}
+    if rank == 0 and not args.kernel_only:
+        def timed(fn, n=5):
+            fn()
+            torch.cuda.synchronize()
+            s, e = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            s.record()
+            for _ in range(n):
+                fn()
+            e.record()
+            torch.cuda.synchronize()
+            return s.elapsed_time(e) / n
+        f16 = dict(dtype=torch.float16, device=dev)
+        Ahi, Alo = torch.empty((M, K), **f16), torch.empty((M, K), **f16)
+        Bhi, Blo = torch.empty((K, N), **f16), torch.empty((K, N), **f16)
+        t_split = timed(lambda: h.sgemm_cube_split(A, Ahi, Alo, SCALE_EXP))
+        h.sgemm_cube_split(B, Bhi, Blo, SCALE_EXP)
+        t_pre = timed(lambda: h.sgemm_cube_presplit(Ahi, Alo, Bhi, Blo, C, SCALE_EXP, binding.TERMWISE))
+        t_unf = timed(lambda: h.sgemm_cube_unfused(A, B, C, SCALE_EXP, binding.TERMWISE))
+        t_ele = timed(lambda: h.sgemm_cube(A, B, C, SCALE_EXP, binding.ELEMENTWISE))
+        extra = {"presplit_kernel_tflops": flops / t_pre / 1e9,
+                 "unfused_split_3gemm_tflops": flops / t_unf / 1e9,
+                 "fused_elementwise_tflops": flops / t_ele / 1e9,
+                 "split_kernel_gbs": 8.0 * M * K / t_split / 1e6}
+        del Ahi, Alo, Bhi, Blo
+
+    if args.kernel_only:
+        if rank == 0:
+            print(json.dumps({"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world,
+                              "steps": args.steps, "ms_per_step": ms_per_step,
+                              "config": {"workload": WORKLOAD}, "kernel_only": True,
+                              "gpu_launches": int(launches)}))
+        h.destroy()
+        if world > 1:
+            dist.destroy_process_group()
+        return
+
+    # End to end through the host-buffer entry point: H2D of A and B, kernel, D2H of C per step.
+    A_pin, B_pin = A_host.pin_memory(), B_host.pin_memory()
+    C_pin = torch.empty((M, N)).pin_memory()
+    h.sgemm_cube_host(A_pin, B_pin, C_pin, SCALE_EXP, binding.TERMWISE)
+    barrier()
+    t0 = time.perf_counter()
+    for _ in range(args.e2e_steps):
+        h.sgemm_cube_host(A_pin, B_pin, C_pin, SCALE_EXP, binding.TERMWISE)
+    barrier()
+    e2e_s = torch.tensor([(time.perf_counter() - t0) / args.e2e_steps], device=dev, dtype=torch.float64)
+    if world > 1:
+        dist.all_reduce(e2e_s, op=dist.ReduceOp.MAX)
+    e2e_val = world * flops / float(e2e_s.item()) / 1e12
+    loss_probe = float(C_pin[0, 0])          # the step's result is read on the host
+
+    if rank == 0:
+        peaks = measured_peaks()
+        kernel_ms = statistics.mean(per_launch_ms)
+        achieved = 3.0 * flops / (kernel_ms * 1e-3) / 1e12      # FP16 tensor-core TFLOP/s
+        peak = peaks["bf16_tflops"]
+        sm_count = torch.cuda.get_device_properties(local_rank).multi_processor_count
+        sm_max = clocks.get("sm_max_mhz") or 1965.0
+        clock_peak = sm_count * 8192 * sm_max * 1e6 / 1e12       # dense FP16 flop/clk/SM x clock
+        cpu_val, cpu_s, cpu_threads = cpu_oracle_sample(args.cpu_rows)
+        out = {
+            "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
+            "warmup": warmup, "ms_per_step": ms_per_step, "higher_is_better": True,
+            "scaling": "weak", "vs_baseline": None, "dtype": "f16 products, f32 accumulate",
+            "data": "synthetic",
+            "config": {"workload": WORKLOAD, "entry_point": "sgemm_cube (fused kernel)",
+                       "l2": "inputs (512 MiB) larger than L2; no flush",
+                       "parallelism": "replicas x%d" % world if world > 1 else "1 GPU"},
+            "clocks": clocks,
+            "e2e": {"value": e2e_val, "unit": UNIT, "h2d_bytes_per_step": 4 * (M * K + K * N),
+                    "d2h_bytes_per_step": 4 * M * N, "result_probe": loss_probe},
+            "gpu_launches": int(launches),
+            "roofline": {"bound": "tensor", "achieved": achieved, "peak": peak, "unit": "TFLOP/s",
+                         "frac": achieved / peak, "traffic": FUSED_KERNEL_DRAM_BYTES_PER_LAUNCH,
+                         "peak_source": "%s cuBLAS bf16 burst (fp16 has the same nominal rate)"
+                                        % peaks["source"],
+                         "kernel_ms": kernel_ms,
+                         "frac_of_sustained": achieved / peaks["bf16_tflops_sustained"],
+                         "frac_of_max_clock_peak": achieved / clock_peak,
+                         "max_clock_peak_tflops": clock_peak},
+            "three_gemm_roofline": {"fp32_equiv_peak_max_clock": clock_peak / 3.0,
+                                    "frac": value / world / (clock_peak / 3.0),
+                                    "fp32_equiv_measured_burst": peak / 3.0,
+                                    "frac_of_measured_burst": value / world / (peak / 3.0)},
+            "cpu_baseline": {"value": cpu_val, "unit": UNIT, "cores": cpu_threads, "kind": "oracle",
+                             "sample": "%d of %d rows of A against the full B, %.1f s"
+                                       % (args.cpu_rows, M, cpu_s)},
+            "ablation": extra,
+            "paper_context": "65.3 TFLOP/s = 77% of 256/3 on Ascend 910A (other hardware; not a target)",
+        }
+        print(json.dumps(out))
+    h.destroy()
+    if world > 1:
+        dist.destroy_process_group()
+
+
+if __name__ == "__main__":
+    main()

@@ -46,7 +46,8 @@ enum {
   SGEMM_CUBE_CUDA_ERROR = 3,       /* a CUDA runtime or driver call failed                      */
   SGEMM_CUBE_DEVICE_TIMEOUT = 4,   /* a kernel gave up on a bounded wait (see sgemm_cube_check) */
   SGEMM_CUBE_UNSUPPORTED_ARCH = 5, /* device is not compute capability 10.x                     */
-  SGEMM_CUBE_ALLOC_FAILED = 6      /* workspace allocation failed                               */
+  SGEMM_CUBE_ALLOC_FAILED = 6,     /* workspace allocation failed                               */
+  SGEMM_CUBE_TOO_LARGE = 7         /* problem exceeds the fixed scratch of the _static variant  */
 };
 
 /* accumulation order (paper Sec. 4.5) */
@@ -156,6 +157,41 @@ int sgemm_cube_host(sgemm_cube_handle h, int M, int N, int K,
                     const float* B_host, int64_t ldb,
                     float* C_host, int64_t ldc,
                     int scale_exp, int accumulation_order, void* stream);
+
+/* Size in bytes of the fixed device scratch area used by sgemm_cube_unfused_static. */
+#define SGEMM_CUBE_STATIC_SCRATCH_BYTES (32u << 20)
+
+/* The unfused computation (same arithmetic, same kernels and same result as sgemm_cube_unfused,
+ * termwise order) for callers that are not allowed to allocate device memory: code running inside
+ * another framework's memory pool with a hard cap, real-time or safety-certified loops where
+ * cudaMalloc/cudaFree (which may synchronise the whole device or fail late) are forbidden after
+ * start-up, or a process whose remaining device memory is already committed.  The paper has no
+ * counterpart of this entry point; it exists for such integrations only.
+ *
+ * It needs no handle and calls no cudaMalloc, cudaFree or other allocating routine.  Its scratch
+ * (the FP16 words of A and B and two FP32 M x N partial results) lives in a fixed array of
+ * SGEMM_CUBE_STATIC_SCRATCH_BYTES (32 MiB) that is part of the library's device image: every GPU
+ * on which the library is loaded holds those 32 MiB until the process exits.
+ *   Limit: 4*(M*K8 + K*N8) + 8*M*N4 bytes (K8, N8 = K, N rounded up to 8; N4 = N rounded up to 4;
+ *   each of the six pieces rounded up to 256 bytes) must not exceed the array, e.g. up to
+ *   1024 x 1024 x 1024 or 2048 x 512 x 1024.  Larger problems return SGEMM_CUBE_TOO_LARGE and
+ *   enqueue nothing.
+ *   Arguments, layouts and alignment as sgemm_cube_unfused, on the CURRENT device
+ *   (A_dev, B_dev, C_dev must be on it).
+ *   The first call on a device looks up the array's device address and configures the kernels;
+ *   make that first call outside any stream capture.  Later calls only launch.
+ *   All calls share the one array, which keeps whatever the last call left in it.  Every region a
+ *   call reads is first overwritten by that call, so results never depend on earlier calls; but
+ *   two calls that may overlap on the GPU (different streams without an ordering between them,
+ *   or different host threads) race on the scratch and give undefined results.
+ *   A kernel-side bounded-wait failure (never expected) cannot be reported by this entry point;
+ *   C is then unspecified.
+ * Errors: INVALID_ARG, TOO_LARGE, UNSUPPORTED_ARCH, CUDA_ERROR. */
+int sgemm_cube_unfused_static(int M, int N, int K,
+                              const float* A_dev, int64_t lda,
+                              const float* B_dev, int64_t ldb,
+                              float* C_dev, int64_t ldc,
+                              int scale_exp, void* stream);
 
 /* Synchronise `stream` and report (then clear) the device error word.
  * Returns OK, DEVICE_TIMEOUT (detail in *detail_out if non-NULL: a code naming the wait that

@@ -12,13 +12,14 @@ import torch
 HERE = os.path.dirname(os.path.abspath(__file__))
 LIB_PATH = os.path.join(HERE, "libsgemm_cube.so")
 
-OK, INVALID_ARG, MISALIGNED, CUDA_ERROR, DEVICE_TIMEOUT, UNSUPPORTED_ARCH, ALLOC_FAILED = range(7)
+OK, INVALID_ARG, MISALIGNED, CUDA_ERROR, DEVICE_TIMEOUT, UNSUPPORTED_ARCH, ALLOC_FAILED, TOO_LARGE = range(8)
+STATIC_SCRATCH_BYTES = 32 << 20
 TERMWISE, ELEMENTWISE = 0, 1
 OPT_TERMWISE_K_BLOCK, OPT_ELEMENTWISE_K_BLOCK = 0, 1
 
 EXPORTS = ["sgemm_cube_create", "sgemm_cube_destroy", "sgemm_cube_set_option", "sgemm_cube_split",
            "sgemm_cube", "sgemm_cube_unfused", "sgemm_cube_presplit", "sgemm_cube_hgemm",
-           "sgemm_cube_host", "sgemm_cube_check", "sgemm_cube_launch_count",
+           "sgemm_cube_host", "sgemm_cube_unfused_static", "sgemm_cube_check", "sgemm_cube_launch_count",
            "sgemm_cube_status_string", "sgemm_cube_version"]
 
 _lib = None
@@ -51,6 +52,7 @@ def load():
     lib.sgemm_cube_presplit.argtypes = [vp, i32, i32, i32, vp, vp, i64, vp, vp, i64, vp, i64, i32,
                                         i32, vp]
     lib.sgemm_cube_hgemm.argtypes = [vp, i32, i32, i32, vp, i64, vp, i64, vp, i64, i32, vp]
+    lib.sgemm_cube_unfused_static.argtypes = [i32, i32, i32, vp, i64, vp, i64, vp, i64, i32, vp]
     lib.sgemm_cube_check.argtypes = [vp, vp, ctypes.POINTER(ctypes.c_uint32)]
     lib.sgemm_cube_launch_count.argtypes = [vp]
     lib.sgemm_cube_launch_count.restype = i64
@@ -91,6 +93,20 @@ def _ld(t):
 def _dev(t, dtype):
     assert t.is_cuda and t.dtype == dtype, "expected a CUDA tensor of dtype %s" % dtype
     return ctypes.c_void_p(t.data_ptr())
+
+
+def sgemm_cube_unfused_static(A, B, C, scale_exp=11, stream=None):
+    """Handle-free, allocation-free variant of Handle.sgemm_cube_unfused for callers that may not
+    allocate device memory: it works out of a fixed 32 MiB scratch area inside the library and
+    therefore only accepts problems that fit it (status TOO_LARGE otherwise).  Runs on the current
+    device; calls that may overlap on the GPU must not be issued (they share the scratch)."""
+    M, K = A.shape
+    K2, N = B.shape
+    assert K == K2 and C.shape == (M, N)
+    _check(load().sgemm_cube_unfused_static(M, N, K, _dev(A, torch.float32), _ld(A),
+                                            _dev(B, torch.float32), _ld(B), _dev(C, torch.float32),
+                                            _ld(C), scale_exp, _stream_ptr(stream)),
+           "sgemm_cube_unfused_static")
 
 
 class Handle:

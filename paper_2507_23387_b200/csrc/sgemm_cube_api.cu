@@ -4,6 +4,7 @@
 #include <cstdio>
 #include <cstdlib>
 #include <cstring>
+#include <mutex>
 #include <new>
 
 #include <cuda.h>
@@ -208,6 +209,7 @@ const char* sgemm_cube_status_string(int status) {
     case SGEMM_CUBE_DEVICE_TIMEOUT: return "a kernel gave up on a bounded wait";
     case SGEMM_CUBE_UNSUPPORTED_ARCH: return "device is not compute capability 10.x (sm_100)";
     case SGEMM_CUBE_ALLOC_FAILED: return "workspace allocation failed";
+    case SGEMM_CUBE_TOO_LARGE: return "problem does not fit the fixed scratch of sgemm_cube_unfused_static";
     default: return "unknown status";
   }
 }
@@ -427,3 +429,113 @@ int sgemm_cube_check(sgemm_cube_handle h, void* stream, uint32_t* detail_out) {
 int64_t sgemm_cube_launch_count(sgemm_cube_handle h) { return h ? h->launches : -1; }
 
 }  // extern "C"
+
+// ---------------------------------------------------------------------------------------------
+// sgemm_cube_unfused_static: the unfused path for callers that must not allocate.
+//
+// Its scratch (the FP16 words of A and B and the two FP32 partial-result matrices) is a fixed
+// array in the library's device image instead of a cudaMalloc'd workspace.  In host code the
+// array's name is only a stand-in: the device address is looked up once per device with
+// cudaGetSymbolAddress while that device is current, and that pointer is what the kernels get.
+namespace {
+
+static __device__ __align__(256) unsigned char g_static_scratch[SGEMM_CUBE_STATIC_SCRATCH_BYTES];
+static __device__ unsigned int g_static_err;
+
+constexpr int kMaxStaticDevices = 64;
+
+struct StaticDeviceState {
+  bool ready = false;
+  unsigned char* scratch = nullptr;   // device address of g_static_scratch on this device
+  sgemm_cube_ctx ctx;                 // host-side launch state; owns no device memory
+};
+
+StaticDeviceState g_static_state[kMaxStaticDevices];
+std::mutex g_static_mutex;
+
+// First call on a device: resolve the device addresses of the scratch array and of the error
+// word, fetch the descriptor encoder and raise the kernels' shared-memory limit.  Allocates nothing.
+int static_setup(int device, StaticDeviceState** out) {
+  if (device < 0 || device >= kMaxStaticDevices) return SGEMM_CUBE_INVALID_ARG;
+  std::lock_guard<std::mutex> lock(g_static_mutex);
+  StaticDeviceState& s = g_static_state[device];
+  if (!s.ready) {
+    int major = 0, sms = 0;
+    if (cudaDeviceGetAttribute(&major, cudaDevAttrComputeCapabilityMajor, device) != cudaSuccess ||
+        cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, device) != cudaSuccess) {
+      cudaGetLastError();
+      return SGEMM_CUBE_CUDA_ERROR;
+    }
+    if (major != 10) return SGEMM_CUBE_UNSUPPORTED_ARCH;
+    void* scratch = nullptr;
+    void* err = nullptr;
+    if (cudaGetSymbolAddress(&scratch, g_static_scratch) != cudaSuccess ||
+        cudaGetSymbolAddress(&err, g_static_err) != cudaSuccess || !scratch || !err) {
+      cudaGetLastError();
+      return SGEMM_CUBE_CUDA_ERROR;
+    }
+    void* fn = nullptr;
+    cudaDriverEntryPointQueryResult qres;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &qres) != cudaSuccess ||
+        qres != cudaDriverEntryPointSuccess || !fn) {
+      cudaGetLastError();
+      return SGEMM_CUBE_CUDA_ERROR;
+    }
+    s.scratch = static_cast<unsigned char*>(scratch);
+    s.ctx.device = device;
+    s.ctx.sm_count = sms;
+    s.ctx.err_dev = static_cast<unsigned int*>(err);
+    s.ctx.encode = reinterpret_cast<EncodeTiledFn>(fn);
+    int rc = set_kernel_attrs(&s.ctx);
+    if (rc) return rc;
+    s.ready = true;
+  }
+  *out = &s;
+  return SGEMM_CUBE_OK;
+}
+
+}  // namespace
+
+extern "C" int sgemm_cube_unfused_static(int M, int N, int K, const float* A, int64_t lda,
+                                         const float* B, int64_t ldb, float* C, int64_t ldc,
+                                         int scale_exp, void* stream) {
+  if (!A || !B || !C) return SGEMM_CUBE_INVALID_ARG;
+  int rc = check_gemm_dims(M, N, K, lda, ldb, ldc);
+  if (rc) return rc;
+  if (scale_exp < 0 || scale_exp > 24) return SGEMM_CUBE_INVALID_ARG;
+  // Same layout as the workspace of sgemm_cube_unfused, carved out of the fixed array.
+  const size_t ldA16 = round_up((size_t)K, 8), ldB16 = round_up((size_t)N, 8);
+  const size_t ldD = round_up((size_t)N, 4);
+  const size_t szA = round_up((size_t)M * ldA16 * 2, 256), szB = round_up((size_t)K * ldB16 * 2, 256);
+  const size_t szD = round_up((size_t)M * ldD * 4, 256);
+  if (2 * szA + 2 * szB + 2 * szD > (size_t)SGEMM_CUBE_STATIC_SCRATCH_BYTES) return SGEMM_CUBE_TOO_LARGE;
+  int device = -1;
+  if (cudaGetDevice(&device) != cudaSuccess) { cudaGetLastError(); return SGEMM_CUBE_CUDA_ERROR; }
+  StaticDeviceState* s = nullptr;
+  rc = static_setup(device, &s);
+  if (rc) return rc;
+  sgemm_cube_ctx* h = &s->ctx;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  unsigned char* w = s->scratch;
+  uint16_t* Ahi = reinterpret_cast<uint16_t*>(w);
+  uint16_t* Alo = reinterpret_cast<uint16_t*>(w + szA);
+  uint16_t* Bhi = reinterpret_cast<uint16_t*>(w + 2 * szA);
+  uint16_t* Blo = reinterpret_cast<uint16_t*>(w + 2 * szA + szB);
+  float* Dhh = reinterpret_cast<float*>(w + 2 * szA + 2 * szB);
+  float* Dx = reinterpret_cast<float*>(w + 2 * szA + 2 * szB + szD);
+  const float inv = ldexpf(1.0f, -scale_exp);
+  const int kb = h->kblock_termwise;
+  // Every region used below is fully overwritten before it is read (D_x by the second pass before
+  // the third adds to it), so nothing left by an earlier call can leak into this one.
+  if ((rc = launch_split(h, M, K, A, lda, Ahi, Alo, (int64_t)ldA16, scale_exp, st))) return rc;
+  if ((rc = launch_split(h, K, N, B, ldb, Bhi, Blo, (int64_t)ldB16, scale_exp, st))) return rc;
+  if ((rc = launch_tc_gemm<1>(h, M, N, K, Ahi, nullptr, ldA16, Bhi, nullptr, ldB16, Dhh, ldD, 0, 0, kb, 1.f, st))) return rc;
+  if ((rc = launch_tc_gemm<1>(h, M, N, K, Alo, nullptr, ldA16, Bhi, nullptr, ldB16, Dx, ldD, 0, 0, kb, 1.f, st))) return rc;
+  if ((rc = launch_tc_gemm<1>(h, M, N, K, Ahi, nullptr, ldA16, Blo, nullptr, ldB16, Dx, ldD, 1, 0, kb, 1.f, st))) return rc;
+  const long long total = (long long)M * N;
+  long long blocks = (total + 255) / 256;
+  const long long cap = (long long)h->sm_count * 16;
+  if (blocks > cap) blocks = cap;
+  sgc::combine_kernel<<<(unsigned)blocks, 256, 0, st>>>(M, N, Dhh, Dx, (long long)ldD, C, ldc, inv);
+  return cudaGetLastError() == cudaSuccess ? SGEMM_CUBE_OK : SGEMM_CUBE_CUDA_ERROR;
+}

@@ -60,6 +60,17 @@ enum : unsigned int {
   kErrConvEmptyWait = 0x106,
 };
 
+// Optional role timing (compile with -DSGC_ROLE_TIMING): CTA 0 adds the clocks each role spends in
+// its phases to a global table; used only for performance investigations.
+#ifdef SGC_ROLE_TIMING
+__device__ unsigned long long g_role_timing[16];
+#define SGC_T0() const long long sgc_t0_ = clock64()
+#define SGC_TADD(slot, cond) do { if (cond) atomicAdd(&g_role_timing[slot], (unsigned long long)(clock64() - sgc_t0_)); } while (0)
+#else
+#define SGC_T0() do {} while (0)
+#define SGC_TADD(slot, cond) do {} while (0)
+#endif
+
 struct TcGemmParams {
   int M, N, K;
   float* D;             // output (C for NTERMS == 3)
@@ -140,13 +151,53 @@ __device__ __forceinline__ void split_pair(float x0, float x1, float scale, uint
   lo2 = *reinterpret_cast<const uint32_t*>(&l);
 }
 
-__device__ __forceinline__ void convert_store(const ConvItem& it, float scale, uint32_t hi_addr,
-                                              uint32_t lo_addr) {
+// Same words with fewer instructions, for s <= 15 (2^s representable in FP16):
+//   xs = x * 2^s            one packed FP32x2 multiply for the pair (exact)
+//   t  = hi * (-2^s) + xs   one mixed-precision FMA per element (FP16 x FP16 + FP32): the exact value
+//                           (x - hi) * 2^s is representable, so the single rounding changes nothing
+// which avoids widening hi to FP32 and the separate subtraction.  (For |x| >= 2^(128-s), outside
+// the method's range, xs overflows and lo becomes NaN where the plain form gives inf.)
+__device__ __forceinline__ void split_pair_fast(float x0, float x1, uint64_t scale2,
+                                                uint16_t neg_scale_h, uint32_t& hi2, uint32_t& lo2) {
+  uint32_t h;
+  asm("cvt.rn.f16x2.f32 %0, %1, %2;" : "=r"(h) : "f"(x1), "f"(x0));
+  uint64_t xp, xs;
+  asm("mov.b64 %0, {%1, %2};" : "=l"(xp) : "f"(x0), "f"(x1));
+  asm("mul.rn.f32x2 %0, %1, %2;" : "=l"(xs) : "l"(xp), "l"(scale2));
+  float xs0, xs1, t0, t1;
+  asm("mov.b64 {%0, %1}, %2;" : "=f"(xs0), "=f"(xs1) : "l"(xs));
+  uint16_t h0, h1;
+  asm("mov.b32 {%0, %1}, %2;" : "=h"(h0), "=h"(h1) : "r"(h));
+  asm("fma.rn.f32.f16 %0, %1, %2, %3;" : "=f"(t0) : "h"(h0), "h"(neg_scale_h), "f"(xs0));
+  asm("fma.rn.f32.f16 %0, %1, %2, %3;" : "=f"(t1) : "h"(h1), "h"(neg_scale_h), "f"(xs1));
+  uint32_t l;
+  asm("cvt.rn.f16x2.f32 %0, %1, %2;" : "=r"(l) : "f"(t1), "f"(t0));
+  hi2 = h;
+  lo2 = l;
+}
+
+struct ConvScale {
+  float scale;            // 2^s
+  uint64_t scale2;        // {2^s, 2^s} packed
+  uint16_t neg_scale_h;   // -2^s as FP16 (valid when fast)
+  bool fast;              // s <= 15
+};
+
+__device__ __forceinline__ void convert_store(const ConvItem& it, const ConvScale& cs,
+                                              uint32_t hi_addr, uint32_t lo_addr) {
   uint4 h, l;
-  split_pair(it.a.x, it.a.y, scale, h.x, l.x);
-  split_pair(it.a.z, it.a.w, scale, h.y, l.y);
-  split_pair(it.b.x, it.b.y, scale, h.z, l.z);
-  split_pair(it.b.z, it.b.w, scale, h.w, l.w);
+  if (cs.fast) {
+    split_pair_fast(it.a.x, it.a.y, cs.scale2, cs.neg_scale_h, h.x, l.x);
+    split_pair_fast(it.a.z, it.a.w, cs.scale2, cs.neg_scale_h, h.y, l.y);
+    split_pair_fast(it.b.x, it.b.y, cs.scale2, cs.neg_scale_h, h.z, l.z);
+    split_pair_fast(it.b.z, it.b.w, cs.scale2, cs.neg_scale_h, h.w, l.w);
+  } else {
+    const float scale = cs.scale;
+    split_pair(it.a.x, it.a.y, scale, h.x, l.x);
+    split_pair(it.a.z, it.a.w, scale, h.y, l.y);
+    split_pair(it.b.x, it.b.y, scale, h.z, l.z);
+    split_pair(it.b.z, it.b.w, scale, h.w, l.w);
+  }
   asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(hi_addr), "r"(h.x), "r"(h.y),
                "r"(h.z), "r"(h.w) : "memory");
   asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(lo_addr), "r"(l.x), "r"(l.y),
@@ -253,8 +304,13 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA0, const __grid_constant__
       for (int c = 0; c < num_chunks && ok; ++c, ++gchunk) {
         const int r_main = (NTERMS == 1) ? (int)(gchunk & 1) : 0;
         const bool with_x = (NTERMS == 3) && (p.order == 1);
-        if (!mbar_wait_bounded(&tfull_bar[r_main], drains[r_main] & 1, abort_flag, p.err,
-                               kErrEpiTmemFullWait)) { ok = false; break; }
+        {
+          SGC_T0();
+          if (!mbar_wait_bounded(&tfull_bar[r_main], drains[r_main] & 1, abort_flag, p.err,
+                                 kErrEpiTmemFullWait)) { ok = false; break; }
+          SGC_TADD(6, blockIdx.x == 0 && threadIdx.x == 0);
+        }
+        SGC_T0();
         if (with_x && !mbar_wait_bounded(&tfull_bar[1], drains[1] & 1, abort_flag, p.err,
                                          kErrEpiTmemFullWait)) { ok = false; break; }
         tc_fence_after_sync();
@@ -289,8 +345,10 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA0, const __grid_constant__
         }
         drains[r_main]++;
         if (with_x) drains[1]++;
+        SGC_TADD(7, blockIdx.x == 0 && threadIdx.x == 0);
       }
       if (!ok) break;
+      SGC_T0();
       const int row = tm * kBM + quarter * 32 + lane;
       const int col_base = tn * kBN + half * 128;
       if (NTERMS == 3 && p.order == 0) {
@@ -319,6 +377,7 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA0, const __grid_constant__
       for (int g = 0; g < 8; ++g)
         store16(p.D, p.ldd, p.M, p.N, row, col_base + g * 16, &S[g * 16], vec_ok,
                 (NTERMS == 1) ? p.accumulate : 0);
+      SGC_TADD(8, blockIdx.x == 0 && threadIdx.x == 0);
     }
   } else if (warp == kMmaWarp) {
     if (FUSED) setmaxnreg_dec<88>();
@@ -344,9 +403,13 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA0, const __grid_constant__
           for (int kb = kb_begin; kb < kb_end && ok; ++kb, ++it) {
             const int s = it % STAGES;
             const uint32_t ph = (it / STAGES) & 1;
-            if (!mbar_wait_bounded(&full_bar[s], ph, abort_flag, p.err, kErrMmaFullWait)) {
-              ok = false;
-              break;
+            {
+              SGC_T0();
+              if (!mbar_wait_bounded(&full_bar[s], ph, abort_flag, p.err, kErrMmaFullWait)) {
+                ok = false;
+                break;
+              }
+              SGC_TADD(4, blockIdx.x == 0);
             }
             tc_fence_after_sync();
             const uint32_t st = smem_u32(smem + s * Cfg::STAGE_BYTES);
@@ -379,8 +442,10 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA0, const __grid_constant__
               }
             }
             if (!main_ready) {
+              SGC_T0();
               if (!mbar_wait_bounded(&tempty_bar[r_main], (fills[r_main] & 1) ^ 1, abort_flag, p.err,
                                      kErrMmaTmemEmptyWait)) { ok = false; break; }
+              SGC_TADD(5, blockIdx.x == 0);
               tc_fence_after_sync();
               main_ready = true;
             }
@@ -464,26 +529,18 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA0, const __grid_constant__
     //   A item -> byte offset m * 64 + ((q ^ ((m >> 1) & 3)) << 4) in the hi/lo A tile (64-byte swizzle)
     //   B item -> atom (c / 8) * 4096 + k * 128 + (((c % 8) ^ (k % 8)) << 4) in the hi/lo B tile
     constexpr int kRounds = 7;
-    constexpr uint32_t kInvalid = 0xFFFFFFFFu;
     const int ct = threadIdx.x - kNumEpiWarps * 32;
-    uint32_t soff[kRounds];     // byte offset of the item's hi chunk inside the stage
-    uint32_t goff[kRounds];     // element offset of the item from the tile's first element
-#pragma unroll
-    for (int r = 0; r < kRounds; ++r) {
-      const int id = ct + r * kConvThreads;
+    const int lda = (int)p.lda32, ldb = (int)p.ldb32;
+    // Geometry of item `id`, recomputed where it is used (keeping 14 offsets per thread alive next
+    // to 56 data registers costs more than these few integer operations).
+    auto smem_off = [&](int id) -> uint32_t {       // byte offset of the hi chunk inside the stage
       if (id < 512) {
         const int m = id >> 2, q = id & 3;
-        soff[r] = (uint32_t)(m * 64 + ((q ^ ((m >> 1) & 3)) << 4));
-        goff[r] = (uint32_t)(m * (int)p.lda32 + q * 8);
-      } else if (id < 1536) {
-        const int b = id - 512, k = b >> 5, c = b & 31;
-        soff[r] = 2 * Cfg::A_TILE + (uint32_t)((c >> 3) * (BK * 128) + k * 128 + (((c & 7) ^ (k & 7)) << 4));
-        goff[r] = (uint32_t)(k * (int)p.ldb32 + c * 8);
-      } else {
-        soff[r] = kInvalid;
-        goff[r] = 0;
+        return (uint32_t)(m * 64 + ((q ^ ((m >> 1) & 3)) << 4));
       }
-    }
+      const int b = id - 512, k = b >> 5, c = b & 31;
+      return 2 * Cfg::A_TILE + (uint32_t)((c >> 3) * (BK * 128) + k * 128 + (((c & 7) ^ (k & 7)) << 4));
+    };
     const int total_stages = ((num_tiles - (int)blockIdx.x + (int)gridDim.x - 1) / (int)gridDim.x) * num_kb;
     ConvItem item[kRounds];
     // Coordinates of the stage whose FP32 data is being loaded (one stage ahead of conversion).
@@ -491,27 +548,37 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA0, const __grid_constant__
     if (ld_tile < num_tiles) tile_coords(ld_tile, num_m, num_n, ld_tm, ld_tn);
     auto load_round = [&](int r) {
       const int id = ct + r * kConvThreads;
+      if (id >= 1536) return;
       const int m0 = ld_tm * kBM, n0 = ld_tn * kBN, k0 = ld_kb * BK;
       const bool interior = (m0 + kBM <= p.M) && (n0 + kBN <= p.N) && (k0 + BK <= p.K);
-      if (soff[r] == kInvalid) return;
       const bool is_a = id < 512;
+      const int row = is_a ? (id >> 2) : ((id - 512) >> 5);          // tile row (A) / k-row (B)
+      const int col = is_a ? ((id & 3) * 8) : (((id - 512) & 31) * 8);
       if (interior) {
-        const float* org = is_a ? (p.A32 + (long long)m0 * p.lda32 + k0)
-                                : (p.B32 + (long long)k0 * p.ldb32 + n0);
-        const float4* src = reinterpret_cast<const float4*>(org + goff[r]);
-        item[r].a = __ldg(src);
-        item[r].b = __ldg(src + 1);
+        const float* src = is_a ? (p.A32 + (long long)(m0 + row) * lda + (k0 + col))
+                                : (p.B32 + (long long)(k0 + row) * ldb + (n0 + col));
+        // volatile asm: the loads are issued here, one stage ahead of their use.
+        asm volatile("ld.global.nc.v4.f32 {%0, %1, %2, %3}, [%4];"
+                     : "=f"(item[r].a.x), "=f"(item[r].a.y), "=f"(item[r].a.z), "=f"(item[r].a.w)
+                     : "l"(src));
+        asm volatile("ld.global.nc.v4.f32 {%0, %1, %2, %3}, [%4 + 16];"
+                     : "=f"(item[r].b.x), "=f"(item[r].b.y), "=f"(item[r].b.z), "=f"(item[r].b.w)
+                     : "l"(src));
       } else if (is_a) {
-        item[r] = load_item_guarded(p.A32, p.lda32, p.M, p.K, m0 + (id >> 2), k0 + (id & 3) * 8);
+        item[r] = load_item_guarded(p.A32, p.lda32, p.M, p.K, m0 + row, k0 + col);
       } else {
-        const int b = id - 512;
-        item[r] = load_item_guarded(p.B32, p.ldb32, p.K, p.N, k0 + (b >> 5), n0 + (b & 31) * 8);
+        item[r] = load_item_guarded(p.B32, p.ldb32, p.K, p.N, k0 + row, n0 + col);
       }
     };
     if (total_stages > 0) {
 #pragma unroll
       for (int r = 0; r < kRounds; ++r) load_round(r);
     }
+    ConvScale cs;
+    cs.scale = p.scale;
+    cs.fast = p.scale <= 32768.f;
+    asm("mov.b64 %0, {%1, %1};" : "=l"(cs.scale2) : "f"(p.scale));
+    cs.neg_scale_h = __half_as_ushort(__float2half_rn(cs.fast ? -p.scale : -1.f));
     for (int it = 0; it < total_stages; ++it) {
       const int s = it % STAGES;
       const uint32_t ph = (it / STAGES) & 1;
@@ -522,22 +589,38 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA0, const __grid_constant__
         if (ld_tile < num_tiles) tile_coords(ld_tile, num_m, num_n, ld_tm, ld_tn);
       }
       const bool more = (it + 1 < total_stages);
-      if (!mbar_wait_bounded(&empty_bar[s], ph ^ 1, abort_flag, p.err, kErrConvEmptyWait)) break;
+      const bool timed = (blockIdx.x == 0 && ct == 0);
+      (void)timed;
+      {
+        SGC_T0();
+        if (!mbar_wait_bounded(&empty_bar[s], ph ^ 1, abort_flag, p.err, kErrConvEmptyWait)) break;
+        SGC_TADD(0, timed);
+      }
+      SGC_T0();
       const uint32_t st = smem_u32(smem + s * Cfg::STAGE_BYTES);
       // Convert the items loaded one stage ago; reload each register set as soon as it is free,
       // so that about one stage of FP32 data per thread is always in flight.
 #pragma unroll
       for (int r = 0; r < kRounds; ++r) {
-        if (soff[r] != kInvalid) {
-          const uint32_t lo_delta = (ct + r * kConvThreads < 512) ? Cfg::A_TILE : Cfg::B_TILE;
-          convert_store(item[r], p.scale, st + soff[r], st + soff[r] + lo_delta);
+        const int id = ct + r * kConvThreads;
+        if (id < 1536) {
+          const uint32_t hi_addr = st + smem_off(id);
+          convert_store(item[r], cs, hi_addr, hi_addr + ((id < 512) ? Cfg::A_TILE : Cfg::B_TILE));
           if (more) load_round(r);
         }
       }
+      SGC_TADD(1, timed);
       // Generic-proxy stores must be visible to the tensor core (async proxy) before the hand-over.
-      fence_proxy_async_smem();
-      __syncwarp();
-      if (lane == 0) mbar_arrive(&full_bar[s]);
+      {
+        SGC_T0();
+        fence_proxy_async_smem();
+        __syncwarp();
+        if (lane == 0) mbar_arrive(&full_bar[s]);
+        SGC_TADD(2, timed);
+      }
+#ifdef SGC_ROLE_TIMING
+      if (timed) atomicAdd(&g_role_timing[3], 1ull);
+#endif
     }
   }
 

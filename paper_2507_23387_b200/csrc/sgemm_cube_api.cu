@@ -539,3 +539,15 @@ extern "C" int sgemm_cube_unfused_static(int M, int N, int K, const float* A, in
   sgc::combine_kernel<<<(unsigned)blocks, 256, 0, st>>>(M, N, Dhh, Dx, (long long)ldD, C, ldc, inv);
   return cudaGetLastError() == cudaSuccess ? SGEMM_CUBE_OK : SGEMM_CUBE_CUDA_ERROR;
 }
+
+#ifdef SGC_ROLE_TIMING
+// Debug builds only: read and clear the role-timing table of tc_gemm_kernel.
+extern "C" int sgemm_cube_debug_role_timing(unsigned long long* out16) {
+  if (cudaDeviceSynchronize() != cudaSuccess) return SGEMM_CUBE_CUDA_ERROR;
+  if (cudaMemcpyFromSymbol(out16, sgc::g_role_timing, 16 * sizeof(unsigned long long)) != cudaSuccess)
+    return SGEMM_CUBE_CUDA_ERROR;
+  unsigned long long z[16] = {0};
+  cudaMemcpyToSymbol(sgc::g_role_timing, z, sizeof(z));
+  return SGEMM_CUBE_OK;
+}
+#endif

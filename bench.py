@@ -156,6 +156,8 @@ def main():
     ap.add_argument("--cpu-rows", type=int, default=2048)
     ap.add_argument("--size", type=int, default=8192,
                     help="M = N = K; values other than 8192 are for profiler captures only")
+    ap.add_argument("--entry", default="sgemm_cube", choices=["sgemm_cube", "presplit", "unfused"],
+                    help="entry point timed as the step (profiler captures; the bench value is sgemm_cube)")
     ap.add_argument("--kernel-only", action="store_true",
                     help="skip the ablation, end-to-end and CPU legs (profiler captures)")
     args = ap.parse_args()
@@ -197,8 +199,24 @@ def main():
             dist.barrier()
         torch.cuda.synchronize()
 
+    if args.entry == "presplit":
+        f16 = dict(dtype=torch.float16, device=dev)
+        pAhi, pAlo = torch.empty((M, K), **f16), torch.empty((M, K), **f16)
+        pBhi, pBlo = torch.empty((K, N), **f16), torch.empty((K, N), **f16)
+        h.sgemm_cube_split(A, pAhi, pAlo, SCALE_EXP)
+        h.sgemm_cube_split(B, pBhi, pBlo, SCALE_EXP)
+
+        def step():
+            h.sgemm_cube_presplit(pAhi, pAlo, pBhi, pBlo, C, SCALE_EXP, binding.TERMWISE)
+    elif args.entry == "unfused":
+        def step():
+            h.sgemm_cube_unfused(A, B, C, SCALE_EXP, binding.TERMWISE)
+    else:
+        def step():
+            h.sgemm_cube(A, B, C, SCALE_EXP, binding.TERMWISE)
+
     for _ in range(warmup):
-        h.sgemm_cube(A, B, C, SCALE_EXP, binding.TERMWISE)
+        step()
     barrier()
     sampler = ClockSampler(local_rank)
     sampler.start()
@@ -207,7 +225,7 @@ def main():
     barrier()
     ev[0].record()
     for i in range(args.steps):
-        h.sgemm_cube(A, B, C, SCALE_EXP, binding.TERMWISE)
+        step()
         ev[i + 1].record()
     barrier()
     total_ms = ev[0].elapsed_time(ev[-1])
@@ -256,7 +274,7 @@ def main():
         if rank == 0:
             print(json.dumps({"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world,
                               "steps": args.steps, "ms_per_step": ms_per_step,
-                              "config": {"workload": WORKLOAD}, "kernel_only": True,
+                              "config": {"workload": WORKLOAD, "entry": args.entry}, "kernel_only": True,
                               "gpu_launches": int(launches)}))
         h.destroy()
         if world > 1:

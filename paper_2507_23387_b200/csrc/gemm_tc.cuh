@@ -531,6 +531,8 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA0, const __grid_constant__
     constexpr int kRounds = 7;
     const int ct = threadIdx.x - kNumEpiWarps * 32;
     const int lda = (int)p.lda32, ldb = (int)p.ldb32;
+    const bool wide_loads = ((lda | ldb) & 7) == 0 &&
+                            (((reinterpret_cast<uintptr_t>(p.A32) | reinterpret_cast<uintptr_t>(p.B32)) & 31) == 0);
     // Geometry of item `id`, recomputed where it is used (keeping 14 offsets per thread alive next
     // to 56 data registers costs more than these few integer operations).
     auto smem_off = [&](int id) -> uint32_t {       // byte offset of the hi chunk inside the stage
@@ -557,13 +559,21 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA0, const __grid_constant__
       if (interior) {
         const float* src = is_a ? (p.A32 + (long long)(m0 + row) * lda + (k0 + col))
                                 : (p.B32 + (long long)(k0 + row) * ldb + (n0 + col));
-        // volatile asm: the loads are issued here, one stage ahead of their use.
-        asm volatile("ld.global.nc.v4.f32 {%0, %1, %2, %3}, [%4];"
-                     : "=f"(item[r].a.x), "=f"(item[r].a.y), "=f"(item[r].a.z), "=f"(item[r].a.w)
-                     : "l"(src));
-        asm volatile("ld.global.nc.v4.f32 {%0, %1, %2, %3}, [%4 + 16];"
-                     : "=f"(item[r].b.x), "=f"(item[r].b.y), "=f"(item[r].b.z), "=f"(item[r].b.w)
-                     : "l"(src));
+        // volatile asm: the loads are issued here, one stage ahead of their use.  One 256-bit
+        // load per item when the rows are 32-byte aligned (a warp then reads 1 KB contiguously).
+        if (wide_loads) {
+          asm volatile("ld.global.nc.v8.f32 {%0, %1, %2, %3, %4, %5, %6, %7}, [%8];"
+                       : "=f"(item[r].a.x), "=f"(item[r].a.y), "=f"(item[r].a.z), "=f"(item[r].a.w),
+                         "=f"(item[r].b.x), "=f"(item[r].b.y), "=f"(item[r].b.z), "=f"(item[r].b.w)
+                       : "l"(src));
+        } else {
+          asm volatile("ld.global.nc.v4.f32 {%0, %1, %2, %3}, [%4];"
+                       : "=f"(item[r].a.x), "=f"(item[r].a.y), "=f"(item[r].a.z), "=f"(item[r].a.w)
+                       : "l"(src));
+          asm volatile("ld.global.nc.v4.f32 {%0, %1, %2, %3}, [%4 + 16];"
+                       : "=f"(item[r].b.x), "=f"(item[r].b.y), "=f"(item[r].b.z), "=f"(item[r].b.w)
+                       : "l"(src));
+        }
       } else if (is_a) {
         item[r] = load_item_guarded(p.A32, p.lda32, p.M, p.K, m0 + row, k0 + col);
       } else {

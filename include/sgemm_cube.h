@@ -64,7 +64,11 @@ enum {
    * of Sec. 4.5 as realised on this hardware. */
   SGEMM_CUBE_OPT_TERMWISE_K_BLOCK = 0,
   /* Same for the elementwise order: the k-block of Eq. elementwise.  Multiple of 64, default 64. */
-  SGEMM_CUBE_OPT_ELEMENTWISE_K_BLOCK = 1
+  SGEMM_CUBE_OPT_ELEMENTWISE_K_BLOCK = 1,
+  /* 1: run the tensor-core kernels as clusters of two CTAs that share one
+   * tcgen05.mma.cta_group::2 (256 x 256 tile per pair, each CTA loading half of the B tile);
+   * 0: one CTA per 128 x 256 tile.  Same arithmetic either way. */
+  SGEMM_CUBE_OPT_CTA_PAIR = 2
 };
 
 /* Create a handle bound to CUDA device `device`.  Allocates a small device error word; the

@@ -88,14 +88,15 @@ struct TcGemmParams {
   float scale;          // 2^s
 };
 
-template <int NTERMS>
+template <int NTERMS, bool PAIR = false>
 struct TcCfg {
   static constexpr int BK = (NTERMS == 1) ? 64 : 32;      // k per pipeline stage
-  static constexpr int STAGES = 4;
+  static constexpr int BN_CTA = PAIR ? kBN / 2 : kBN;     // B columns held by one CTA
   static constexpr int A_ROW_BYTES = BK * 2;              // 128 or 64: also the swizzle span of A
   static constexpr uint32_t A_TILE = kBM * BK * 2;        // one FP16 A tile
-  static constexpr uint32_t B_TILE = BK * kBN * 2;        // one FP16 B tile
+  static constexpr uint32_t B_TILE = BK * BN_CTA * 2;     // one FP16 B tile (this CTA's columns)
   static constexpr uint32_t STAGE_BYTES = (NTERMS == 1) ? (A_TILE + B_TILE) : 2 * (A_TILE + B_TILE);
+  static constexpr int STAGES = (196608 / STAGE_BYTES) > 8 ? 8 : (196608 / STAGE_BYTES);
   static constexpr uint32_t SMEM_BYTES = STAGES * STAGE_BYTES + 1024 /*align*/ + 256 /*barriers*/;
 };
 
@@ -224,14 +225,24 @@ __device__ __forceinline__ ConvItem load_item_guarded(const float* __restrict__ 
   return it;
 }
 
-template <int NTERMS, bool FUSED>
+__device__ __forceinline__ void tmem_ld_cols(uint32_t taddr, uint32_t (&r)[16]) { tmem_ld_32x32b_x16(taddr, r); }
+__device__ __forceinline__ void tmem_ld_cols(uint32_t taddr, uint32_t (&r)[32]) { tmem_ld_32x32b_x32(taddr, r); }
+
+template <int NTERMS, bool FUSED, bool PAIR>
 __global__ void __launch_bounds__(FUSED ? kFusedThreads : kTcThreads, 1)
 tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA0, const __grid_constant__ CUtensorMap tmA1,
                const __grid_constant__ CUtensorMap tmB0, const __grid_constant__ CUtensorMap tmB1,
                const TcGemmParams p) {
-  using Cfg = TcCfg<NTERMS>;
+  using Cfg = TcCfg<NTERMS, PAIR>;
   constexpr int BK = Cfg::BK;
   constexpr int STAGES = Cfg::STAGES;
+  // PAIR: the kernel runs as clusters of two CTAs driving tcgen05.mma.cta_group::2.  The pair owns
+  // a 256 x 256 tile: CTA rank r holds rows [128 r, 128 r + 128) of A and of the result (its own
+  // TMEM lanes) and columns [128 r, 128 r + 128) of the B tile; rank 0 (the leader) issues the MMAs
+  // for both, so the "full" and "TMEM drained" barriers that its MMA thread waits on live in the
+  // leader and are signalled by both CTAs, while its commits arrive on the barriers of both.
+  const uint32_t cta_rank = PAIR ? cluster_ctarank() : 0u;
+  const bool leader = (cta_rank == 0);
   constexpr int kProducerWarp = 8;                    // not FUSED
   constexpr int kMmaWarp = FUSED ? 15 : 9;
   static_assert(!FUSED || NTERMS == 3, "the fused kernel computes all three products");
@@ -252,13 +263,24 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA0, const __grid_constant__
 
   const int warp = threadIdx.x >> 5;
   const int lane = threadIdx.x & 31;
+#ifdef SGC_ROLE_TIMING
+  long long sgc_k_clk0 = 0;
+  unsigned long long sgc_k_ns0 = 0;
+  if (blockIdx.x == 0 && threadIdx.x == 0) {
+    sgc_k_clk0 = clock64();
+    asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(sgc_k_ns0));
+  }
+#endif
 
   if (threadIdx.x == 0) {
     for (int s = 0; s < STAGES; ++s) {
-      mbar_init(&full_bar[s], FUSED ? kNumConvWarps : 1);
+      mbar_init(&full_bar[s], FUSED ? kNumConvWarps * (PAIR ? 2 : 1) : 1);
       mbar_init(&empty_bar[s], 1);
     }
-    for (int r = 0; r < 2; ++r) { mbar_init(&tfull_bar[r], 1); mbar_init(&tempty_bar[r], kNumEpiWarps); }
+    for (int r = 0; r < 2; ++r) {
+      mbar_init(&tfull_bar[r], 1);
+      mbar_init(&tempty_bar[r], kNumEpiWarps * (PAIR ? 2 : 1));
+    }
     mbar_init(drain_bar, 1);
     *abort_flag = 0u;
     fence_mbar_init();
@@ -267,18 +289,26 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA0, const __grid_constant__
     tma_prefetch_desc(&tmA0); tma_prefetch_desc(&tmB0);
     if (NTERMS == 3) { tma_prefetch_desc(&tmA1); tma_prefetch_desc(&tmB1); }
   }
-  if (warp == kMmaWarp) {    // whole warp: allocate all 512 TMEM columns
-    tmem_alloc(tmem_base_slot, kTmemCols);
-    tmem_relinquish();
+  if (warp == kMmaWarp) {    // whole warp (the same warp in both CTAs of a pair): all 512 TMEM columns
+    if (PAIR) { tmem_alloc_pair(tmem_base_slot, kTmemCols); tmem_relinquish_pair(); }
+    else { tmem_alloc(tmem_base_slot, kTmemCols); tmem_relinquish(); }
   }
   tc_fence_before_sync();
   __syncthreads();
+  if (PAIR) cluster_sync_all();      // the peer's barriers are initialised before anyone signals them
   tc_fence_after_sync();
   const uint32_t tmem_base = *tmem_base_slot;
 
-  const int num_m = (p.M + kBM - 1) / kBM;
+  // Work units: 128-row tiles, or 256-row pair tiles of which this CTA takes row block `cta_rank`.
+  const int num_m = PAIR ? (p.M + 2 * kBM - 1) / (2 * kBM) : (p.M + kBM - 1) / kBM;
   const int num_n = (p.N + kBN - 1) / kBN;
   const int num_tiles = num_m * num_n;
+  const int first_tile = PAIR ? (int)(blockIdx.x >> 1) : (int)blockIdx.x;
+  const int tile_stride = PAIR ? (int)(gridDim.x >> 1) : (int)gridDim.x;
+  auto tile_rc = [&](int tile, int& tm, int& tn) {     // tm in units of 128 rows, tn of 256 columns
+    tile_coords(tile, num_m, num_n, tm, tn);
+    if (PAIR) tm = tm * 2 + (int)cta_rank;
+  };
   const int num_kb = (p.K + BK - 1) / BK;                      // pipeline stages per tile
   const int chunk = p.kchunk_blocks;                           // stages per k-block g
   const int num_chunks = (num_kb + chunk - 1) / chunk;
@@ -298,50 +328,59 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA0, const __grid_constant__
     uint32_t gchunk = 0;
     bool ok = true;
     float S[128];
-    for (int tile = blockIdx.x; tile < num_tiles && ok; tile += gridDim.x) {
+    // TMEM is read 32 columns at a time (fewer, longer loads: the load latency is what a drain
+    // costs), 16 where the register budget is tight.
+    constexpr int GW = FUSED ? 16 : 32;
+    auto wait_tfull = [&](int r) -> bool {
+      return mbar_wait_bounded(&tfull_bar[r], drains[r] & 1, abort_flag, p.err, kErrEpiTmemFullWait);
+    };
+    // "TMEM region drained": arrive on the leader's barrier (the peer does so remotely).
+    auto arrive_tempty = [&](int r) {
+      if (!PAIR || leader) mbar_arrive(&tempty_bar[r]);
+      else mbar_arrive_cluster(mapa_u32(smem_u32(&tempty_bar[r]), 0));
+    };
+    for (int tile = first_tile; tile < num_tiles && ok; tile += tile_stride) {
       int tm, tn;
-      tile_coords(tile, num_m, num_n, tm, tn);
+      tile_rc(tile, tm, tn);
       for (int c = 0; c < num_chunks && ok; ++c, ++gchunk) {
         const int r_main = (NTERMS == 1) ? (int)(gchunk & 1) : 0;
         const bool with_x = (NTERMS == 3) && (p.order == 1);
         {
           SGC_T0();
-          if (!mbar_wait_bounded(&tfull_bar[r_main], drains[r_main] & 1, abort_flag, p.err,
-                                 kErrEpiTmemFullWait)) { ok = false; break; }
+          if (!wait_tfull(r_main)) { ok = false; break; }
           SGC_TADD(6, blockIdx.x == 0 && threadIdx.x == 0);
         }
         SGC_T0();
-        if (with_x && !mbar_wait_bounded(&tfull_bar[1], drains[1] & 1, abort_flag, p.err,
-                                         kErrEpiTmemFullWait)) { ok = false; break; }
+        if (with_x && !wait_tfull(1)) { ok = false; break; }
         tc_fence_after_sync();
         const uint32_t t_main = tmem_base + lane_addr + r_main * kBN + half * 128;
         const uint32_t t_x = tmem_base + lane_addr + kBN + half * 128;
 #pragma unroll
-        for (int g = 0; g < 8; ++g) {
-          uint32_t v[16];
-          tmem_ld_32x32b_x16(t_main + g * 16, v);
+        for (int g = 0; g < 128 / GW; ++g) {
+          uint32_t v[GW];
+          tmem_ld_cols(t_main + g * GW, v);
           tmem_ld_wait();
           if (c == 0) {
 #pragma unroll
-            for (int j = 0; j < 16; ++j) S[g * 16 + j] = __uint_as_float(v[j]);
+            for (int j = 0; j < GW; ++j) S[g * GW + j] = __uint_as_float(v[j]);
           } else {
 #pragma unroll
-            for (int j = 0; j < 16; ++j) S[g * 16 + j] = __fadd_rn(S[g * 16 + j], __uint_as_float(v[j]));
+            for (int j = 0; j < GW; ++j) S[g * GW + j] = __fadd_rn(S[g * GW + j], __uint_as_float(v[j]));
           }
           if (with_x) {
             // Elementwise: fold this k-block's corrections into the same accumulator.
-            tmem_ld_32x32b_x16(t_x + g * 16, v);
+            tmem_ld_cols(t_x + g * GW, v);
             tmem_ld_wait();
 #pragma unroll
-            for (int j = 0; j < 16; ++j)
-              S[g * 16 + j] = __fadd_rn(S[g * 16 + j], __fmul_rn(__uint_as_float(v[j]), p.inv_scale));
+            for (int j = 0; j < GW; ++j)
+              S[g * GW + j] = __fadd_rn(S[g * GW + j], __fmul_rn(__uint_as_float(v[j]), p.inv_scale));
           }
         }
         tc_fence_before_sync();
         __syncwarp();
         if (lane == 0) {
-          mbar_arrive(&tempty_bar[r_main]);
-          if (with_x) mbar_arrive(&tempty_bar[1]);
+          arrive_tempty(r_main);
+          if (with_x) arrive_tempty(1);
         }
         drains[r_main]++;
         if (with_x) drains[1]++;
@@ -353,24 +392,24 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA0, const __grid_constant__
       const int col_base = tn * kBN + half * 128;
       if (NTERMS == 3 && p.order == 0) {
         // Termwise: the correction stream meets the dominant stream once, here.
-        if (!mbar_wait_bounded(&tfull_bar[1], drains[1] & 1, abort_flag, p.err, kErrEpiTmemFullWait)) {
+        if (!wait_tfull(1)) {
           ok = false;
           break;
         }
         tc_fence_after_sync();
         const uint32_t t_x = tmem_base + lane_addr + kBN + half * 128;
 #pragma unroll
-        for (int g = 0; g < 8; ++g) {
-          uint32_t v[16];
-          tmem_ld_32x32b_x16(t_x + g * 16, v);
+        for (int g = 0; g < 128 / GW; ++g) {
+          uint32_t v[GW];
+          tmem_ld_cols(t_x + g * GW, v);
           tmem_ld_wait();
 #pragma unroll
-          for (int j = 0; j < 16; ++j)
-            S[g * 16 + j] = __fadd_rn(S[g * 16 + j], __fmul_rn(__uint_as_float(v[j]), p.inv_scale));
+          for (int j = 0; j < GW; ++j)
+            S[g * GW + j] = __fadd_rn(S[g * GW + j], __fmul_rn(__uint_as_float(v[j]), p.inv_scale));
         }
         tc_fence_before_sync();
         __syncwarp();
-        if (lane == 0) mbar_arrive(&tempty_bar[1]);
+        if (lane == 0) arrive_tempty(1);
         drains[1]++;
       }
 #pragma unroll
@@ -382,8 +421,21 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA0, const __grid_constant__
   } else if (warp == kMmaWarp) {
     if (FUSED) setmaxnreg_dec<88>();
     // ------------------------------------------------------------------ MMA issuer
-    if (lane == 0) {
-      constexpr uint32_t idesc = umma_idesc_f16(kBM, kBN, /*A MN-major*/ false, /*B MN-major*/ true);
+    if (lane == 0 && leader) {
+      constexpr uint32_t idesc =
+          umma_idesc_f16(PAIR ? 2 * kBM : kBM, kBN, /*A MN-major*/ false, /*B MN-major*/ true);
+      auto mma = [&](uint32_t d, uint64_t da, uint64_t db, uint32_t acc) {
+        if (PAIR) umma_f16_ss_pair(d, da, db, idesc, acc);
+        else umma_f16_ss(d, da, db, idesc, acc);
+      };
+      auto commit_both = [&](uint64_t* bar) {            // barrier at this offset in every CTA
+        if (PAIR) umma_commit_pair_both(bar);
+        else umma_commit(bar);
+      };
+      auto wait = [&](uint64_t* bar, uint32_t parity, unsigned int code) {
+        return PAIR ? mbar_wait_bounded_cluster(bar, parity, abort_flag, p.err, code)
+                    : mbar_wait_bounded(bar, parity, abort_flag, p.err, code);
+      };
       constexpr uint64_t a_swz = (Cfg::A_ROW_BYTES == 128) ? kSwizzle128 : kSwizzle64;
       constexpr uint32_t a_sbo = 8 * Cfg::A_ROW_BYTES;     // 8 rows of the swizzle atom
       constexpr uint32_t b_lbo = BK * 128;                 // next 64-column atom of B
@@ -392,7 +444,7 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA0, const __grid_constant__
       uint32_t fills[2] = {0, 0};     // how many times each TMEM region has been handed over
       uint32_t gchunk = 0;            // running k-block counter (NTERMS == 1 region choice)
       bool ok = true;
-      for (int tile = blockIdx.x; tile < num_tiles && ok; tile += gridDim.x) {
+      for (int tile = first_tile; tile < num_tiles && ok; tile += tile_stride) {
         for (int c = 0; c < num_chunks && ok; ++c, ++gchunk) {
           const int kb_begin = c * chunk;
           const int kb_end = min(num_kb, kb_begin + chunk);
@@ -400,76 +452,95 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA0, const __grid_constant__
           const int r_main = (NTERMS == 1) ? (int)(gchunk & 1) : 0;
           const bool x_fresh = (NTERMS == 3) && (p.order == 1 || c == 0);
           bool main_ready = false, x_ready = !x_fresh;
-          for (int kb = kb_begin; kb < kb_end && ok; ++kb, ++it) {
-            const int s = it % STAGES;
-            const uint32_t ph = (it / STAGES) & 1;
-            {
-              SGC_T0();
-              if (!mbar_wait_bounded(&full_bar[s], ph, abort_flag, p.err, kErrMmaFullWait)) {
-                ok = false;
-                break;
-              }
-              SGC_TADD(4, blockIdx.x == 0);
-            }
+          const uint32_t d_x = tmem_base + kBN;
+          const uint32_t d_main = tmem_base + r_main * kBN;
+          // Wait for stage `i` (running stage counter) to be filled; returns its base address.
+          auto stage_ready = [&](uint32_t i, uint32_t& st) -> bool {
+            const int s = i % STAGES;
+            SGC_T0();
+            if (!wait(&full_bar[s], (i / STAGES) & 1, kErrMmaFullWait)) return false;
+            SGC_TADD(4, blockIdx.x == 0);
             tc_fence_after_sync();
-            const uint32_t st = smem_u32(smem + s * Cfg::STAGE_BYTES);
-            const uint32_t a_hi = st;
-            const uint32_t a_lo = st + Cfg::A_TILE;
-            const uint32_t b_hi = st + ((NTERMS == 3) ? 2 * Cfg::A_TILE : Cfg::A_TILE);
-            const uint32_t b_lo = b_hi + Cfg::B_TILE;
-            const bool first_kb = (kb == kb_begin);
-            if (NTERMS == 3) {
-              // Correction products first: they do not depend on region 0 being drained, so the
-              // accumulate warps get this time to add the previous k-block into their sums.
-              if (!x_ready) {
-                if (!mbar_wait_bounded(&tempty_bar[1], (fills[1] & 1) ^ 1, abort_flag, p.err,
-                                       kErrMmaTmemEmptyWait)) { ok = false; break; }
-                tc_fence_after_sync();
-                x_ready = true;
-              }
-              const uint32_t d_x = tmem_base + kBN;
-#pragma unroll
-              for (int j = 0; j < BK / 16; ++j) {
-                const uint64_t da = umma_smem_desc(a_lo + j * 32, 16, a_sbo, a_swz);
-                const uint64_t db = umma_smem_desc(b_hi + j * 2048, b_lbo, b_sbo, kSwizzle128);
-                umma_f16_ss(d_x, da, db, idesc, (x_fresh && first_kb && j == 0) ? 0u : 1u);
-              }
-#pragma unroll
-              for (int j = 0; j < BK / 16; ++j) {
-                const uint64_t da = umma_smem_desc(a_hi + j * 32, 16, a_sbo, a_swz);
-                const uint64_t db = umma_smem_desc(b_lo + j * 2048, b_lbo, b_sbo, kSwizzle128);
-                umma_f16_ss(d_x, da, db, idesc, 1u);
-              }
+            st = smem_u32(smem + s * Cfg::STAGE_BYTES);
+            return true;
+          };
+          // lo_A hi_B and hi_A lo_B of one stage into the correction accumulator.
+          auto issue_cross = [&](uint32_t st, bool first_kb) -> bool {
+            if (!x_ready) {
+              if (!wait(&tempty_bar[1], (fills[1] & 1) ^ 1, kErrMmaTmemEmptyWait)) return false;
+              tc_fence_after_sync();
+              x_ready = true;
             }
+            const uint32_t a_hi = st, a_lo = st + Cfg::A_TILE;
+            const uint32_t b_hi = st + 2 * Cfg::A_TILE, b_lo = b_hi + Cfg::B_TILE;
+#pragma unroll
+            for (int j = 0; j < BK / 16; ++j) {
+              const uint64_t da = umma_smem_desc(a_lo + j * 32, 16, a_sbo, a_swz);
+              const uint64_t db = umma_smem_desc(b_hi + j * 2048, b_lbo, b_sbo, kSwizzle128);
+              mma(d_x, da, db, (x_fresh && first_kb && j == 0) ? 0u : 1u);
+            }
+#pragma unroll
+            for (int j = 0; j < BK / 16; ++j) {
+              const uint64_t da = umma_smem_desc(a_hi + j * 32, 16, a_sbo, a_swz);
+              const uint64_t db = umma_smem_desc(b_lo + j * 2048, b_lbo, b_sbo, kSwizzle128);
+              mma(d_x, da, db, 1u);
+            }
+            return true;
+          };
+          // hi_A hi_B (or the single product) of one stage into the main region; frees the stage.
+          auto issue_main = [&](uint32_t st, uint32_t i, bool first_kb) -> bool {
             if (!main_ready) {
               SGC_T0();
-              if (!mbar_wait_bounded(&tempty_bar[r_main], (fills[r_main] & 1) ^ 1, abort_flag, p.err,
-                                     kErrMmaTmemEmptyWait)) { ok = false; break; }
+              if (!wait(&tempty_bar[r_main], (fills[r_main] & 1) ^ 1, kErrMmaTmemEmptyWait)) return false;
               SGC_TADD(5, blockIdx.x == 0);
               tc_fence_after_sync();
               main_ready = true;
             }
-            const uint32_t d_main = tmem_base + r_main * kBN;
+            const uint32_t a_hi = st;
+            const uint32_t b_hi = st + ((NTERMS == 3) ? 2 * Cfg::A_TILE : Cfg::A_TILE);
 #pragma unroll
             for (int j = 0; j < BK / 16; ++j) {
               const uint64_t da = umma_smem_desc(a_hi + j * 32, 16, a_sbo, a_swz);
               const uint64_t db = umma_smem_desc(b_hi + j * 2048, b_lbo, b_sbo, kSwizzle128);
-              umma_f16_ss(d_main, da, db, idesc, (first_kb && j == 0) ? 0u : 1u);
+              mma(d_main, da, db, (first_kb && j == 0) ? 0u : 1u);
             }
-            umma_commit(&empty_bar[s]);          // stage s may be refilled once these MMAs retire
+            commit_both(&empty_bar[i % STAGES]);   // the stage may be refilled once these MMAs retire
+            return true;
+          };
+          int kb = kb_begin;
+          constexpr int kLook = PAIR ? 3 : 2;      // stages whose correction products go first
+          if (NTERMS == 3 && p.order == 0 && kb + kLook <= kb_end) {
+            // Start of a termwise k-block: the correction products of the first kLook stages go
+            // first.  They do not touch region 0, so the accumulate warps get 8 kLook MMAs' worth
+            // of time to add the previous k-block into their sums before hi*hi needs the region.
+            uint32_t st[kLook];
+#pragma unroll
+            for (int l = 0; l < kLook; ++l)
+              ok = ok && stage_ready(it + l, st[l]) && issue_cross(st[l], l == 0);
+#pragma unroll
+            for (int l = 0; l < kLook; ++l) ok = ok && issue_main(st[l], it + l, l == 0);
+            kb += kLook;
+            it += kLook;
+          }
+          for (; kb < kb_end && ok; ++kb, ++it) {
+            uint32_t st;
+            const bool first_kb = (kb == kb_begin);
+            ok = stage_ready(it, st) && (NTERMS != 3 || issue_cross(st, first_kb)) &&
+                 issue_main(st, it, first_kb);
           }
           if (!ok) break;
           // Hand the finished region(s) to the accumulate warps.
-          umma_commit(&tfull_bar[r_main]);
+          commit_both(&tfull_bar[r_main]);
           fills[r_main]++;
           if (NTERMS == 3 && (p.order == 1 || c == num_chunks - 1)) {
-            umma_commit(&tfull_bar[1]);
+            commit_both(&tfull_bar[1]);
             fills[1]++;
           }
         }
       }
       // Bounded drain: all issued MMAs must have retired before TMEM is freed.
-      umma_commit(drain_bar);
+      if (PAIR) umma_commit_pair_local(drain_bar);
+      else umma_commit(drain_bar);
       mbar_wait_bounded(drain_bar, 0, nullptr, p.err, kErrDrainWait);
     }
   } else if (!FUSED) {
@@ -477,9 +548,14 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA0, const __grid_constant__
     if (lane == 0) {
       uint32_t it = 0;
       bool ok = true;
-      for (int tile = blockIdx.x; tile < num_tiles && ok; tile += gridDim.x) {
+      auto load = [&](void* dst, const CUtensorMap* map, int x, int y, uint64_t* bar) {
+        if (PAIR) tma_load_2d_pair(dst, map, x, y, bar);    // bytes counted on the leader's barrier
+        else tma_load_2d(dst, map, x, y, bar);
+      };
+      for (int tile = first_tile; tile < num_tiles && ok; tile += tile_stride) {
         int tm, tn;
-        tile_coords(tile, num_m, num_n, tm, tn);
+        tile_rc(tile, tm, tn);
+        const int n0 = tn * kBN + (PAIR ? (int)cta_rank * Cfg::BN_CTA : 0);   // this CTA's B columns
         for (int kb = 0; kb < num_kb; ++kb, ++it) {
           const int s = it % STAGES;
           const uint32_t ph = (it / STAGES) & 1;
@@ -488,23 +564,24 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA0, const __grid_constant__
             break;
           }
           uint8_t* st = smem + s * Cfg::STAGE_BYTES;
-          mbar_arrive_expect_tx(&full_bar[s], Cfg::STAGE_BYTES);
+          // The leader announces the bytes of both CTAs' copies; the peer's copies may land first
+          // (the phase cannot complete before the leader's arrival).
+          if (leader) mbar_arrive_expect_tx(&full_bar[s], Cfg::STAGE_BYTES * (PAIR ? 2 : 1));
           const int k0 = kb * BK;
-          // A tiles: box {BK (k), 128 rows}.  B tiles: 4 boxes {64 (n), BK (k rows)}.
-          tma_load_2d(st, &tmA0, k0, tm * kBM, &full_bar[s]);
+          // A tiles: box {BK (k), 128 rows}.  B tiles: boxes {64 (n), BK (k rows)}.
+          load(st, &tmA0, k0, tm * kBM, &full_bar[s]);
           uint8_t* bdst = st + Cfg::A_TILE;
           if (NTERMS == 3) {
-            tma_load_2d(st + Cfg::A_TILE, &tmA1, k0, tm * kBM, &full_bar[s]);
+            load(st + Cfg::A_TILE, &tmA1, k0, tm * kBM, &full_bar[s]);
             bdst = st + 2 * Cfg::A_TILE;
           }
 #pragma unroll
-          for (int a = 0; a < kBN / 64; ++a)
-            tma_load_2d(bdst + a * (BK * 128), &tmB0, tn * kBN + a * 64, k0, &full_bar[s]);
+          for (int a = 0; a < Cfg::BN_CTA / 64; ++a)
+            load(bdst + a * (BK * 128), &tmB0, n0 + a * 64, k0, &full_bar[s]);
           if (NTERMS == 3) {
 #pragma unroll
-            for (int a = 0; a < kBN / 64; ++a)
-              tma_load_2d(bdst + Cfg::B_TILE + a * (BK * 128), &tmB1, tn * kBN + a * 64, k0,
-                          &full_bar[s]);
+            for (int a = 0; a < Cfg::BN_CTA / 64; ++a)
+              load(bdst + Cfg::B_TILE + a * (BK * 128), &tmB1, n0 + a * 64, k0, &full_bar[s]);
           }
         }
       }
@@ -528,7 +605,10 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA0, const __grid_constant__
     // coalesced loads and bank-conflict-free 16-byte stores into the swizzled tiles.
     //   A item -> byte offset m * 64 + ((q ^ ((m >> 1) & 3)) << 4) in the hi/lo A tile (64-byte swizzle)
     //   B item -> atom (c / 8) * 4096 + k * 128 + (((c % 8) ^ (k % 8)) << 4) in the hi/lo B tile
-    constexpr int kRounds = 7;
+    // (PAIR: this CTA's B tile is 32 x 128, 512 items, ids 512-1023, 16 chunks per k-row.)
+    constexpr int kChunksPerRow = Cfg::BN_CTA / 8;                 // B chunks per k-row: 32 or 16
+    constexpr int kItems = 512 + BK * kChunksPerRow;               // 1536 or 1024
+    constexpr int kRounds = (kItems + kConvThreads - 1) / kConvThreads;   // 7 or 5
     const int ct = threadIdx.x - kNumEpiWarps * 32;
     const int lda = (int)p.lda32, ldb = (int)p.ldb32;
     const bool wide_loads = ((lda | ldb) & 7) == 0 &&
@@ -540,22 +620,24 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA0, const __grid_constant__
         const int m = id >> 2, q = id & 3;
         return (uint32_t)(m * 64 + ((q ^ ((m >> 1) & 3)) << 4));
       }
-      const int b = id - 512, k = b >> 5, c = b & 31;
+      const int b = id - 512, k = b / kChunksPerRow, c = b % kChunksPerRow;
       return 2 * Cfg::A_TILE + (uint32_t)((c >> 3) * (BK * 128) + k * 128 + (((c & 7) ^ (k & 7)) << 4));
     };
-    const int total_stages = ((num_tiles - (int)blockIdx.x + (int)gridDim.x - 1) / (int)gridDim.x) * num_kb;
+    const int total_stages = (first_tile < num_tiles)
+        ? ((num_tiles - first_tile + tile_stride - 1) / tile_stride) * num_kb : 0;
     ConvItem item[kRounds];
     // Coordinates of the stage whose FP32 data is being loaded (one stage ahead of conversion).
-    int ld_tile = blockIdx.x, ld_kb = 0, ld_tm = 0, ld_tn = 0;
-    if (ld_tile < num_tiles) tile_coords(ld_tile, num_m, num_n, ld_tm, ld_tn);
+    int ld_tile = first_tile, ld_kb = 0, ld_tm = 0, ld_tn = 0;
+    if (ld_tile < num_tiles) tile_rc(ld_tile, ld_tm, ld_tn);
     auto load_round = [&](int r) {
       const int id = ct + r * kConvThreads;
-      if (id >= 1536) return;
-      const int m0 = ld_tm * kBM, n0 = ld_tn * kBN, k0 = ld_kb * BK;
-      const bool interior = (m0 + kBM <= p.M) && (n0 + kBN <= p.N) && (k0 + BK <= p.K);
+      if (id >= kItems) return;
+      const int m0 = ld_tm * kBM, k0 = ld_kb * BK;
+      const int n0 = ld_tn * kBN + (PAIR ? (int)cta_rank * Cfg::BN_CTA : 0);
+      const bool interior = (m0 + kBM <= p.M) && (n0 + Cfg::BN_CTA <= p.N) && (k0 + BK <= p.K);
       const bool is_a = id < 512;
-      const int row = is_a ? (id >> 2) : ((id - 512) >> 5);          // tile row (A) / k-row (B)
-      const int col = is_a ? ((id & 3) * 8) : (((id - 512) & 31) * 8);
+      const int row = is_a ? (id >> 2) : ((id - 512) / kChunksPerRow);     // tile row (A) / k-row (B)
+      const int col = is_a ? ((id & 3) * 8) : (((id - 512) % kChunksPerRow) * 8);
       if (interior) {
         const float* src = is_a ? (p.A32 + (long long)(m0 + row) * lda + (k0 + col))
                                 : (p.B32 + (long long)(k0 + row) * ldb + (n0 + col));
@@ -595,8 +677,8 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA0, const __grid_constant__
       // advance the load coordinates to stage it + 1
       if (++ld_kb == num_kb) {
         ld_kb = 0;
-        ld_tile += gridDim.x;
-        if (ld_tile < num_tiles) tile_coords(ld_tile, num_m, num_n, ld_tm, ld_tn);
+        ld_tile += tile_stride;
+        if (ld_tile < num_tiles) tile_rc(ld_tile, ld_tm, ld_tn);
       }
       const bool more = (it + 1 < total_stages);
       const bool timed = (blockIdx.x == 0 && ct == 0);
@@ -613,7 +695,7 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA0, const __grid_constant__
 #pragma unroll
       for (int r = 0; r < kRounds; ++r) {
         const int id = ct + r * kConvThreads;
-        if (id < 1536) {
+        if (id < kItems) {
           const uint32_t hi_addr = st + smem_off(id);
           convert_store(item[r], cs, hi_addr, hi_addr + ((id < 512) ? Cfg::A_TILE : Cfg::B_TILE));
           if (more) load_round(r);
@@ -623,9 +705,13 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA0, const __grid_constant__
       // Generic-proxy stores must be visible to the tensor core (async proxy) before the hand-over.
       {
         SGC_T0();
-        fence_proxy_async_smem();
+        if (PAIR) fence_proxy_async_all();
+        else fence_proxy_async_smem();
         __syncwarp();
-        if (lane == 0) mbar_arrive(&full_bar[s]);
+        if (lane == 0) {
+          if (!PAIR || leader) mbar_arrive(&full_bar[s]);
+          else mbar_arrive_cluster(mapa_u32(smem_u32(&full_bar[s]), 0));   // the leader's barrier
+        }
         SGC_TADD(2, timed);
       }
 #ifdef SGC_ROLE_TIMING
@@ -637,10 +723,20 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA0, const __grid_constant__
   // ---------------------------------------------------------------------- teardown
   tc_fence_before_sync();
   __syncthreads();
+#ifdef SGC_ROLE_TIMING
+  if (blockIdx.x == 0 && threadIdx.x == 0) {
+    unsigned long long ns1;
+    asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(ns1));
+    atomicAdd(&g_role_timing[9], (unsigned long long)(clock64() - sgc_k_clk0));
+    atomicAdd(&g_role_timing[10], ns1 - sgc_k_ns0);
+  }
+#endif
+  if (PAIR) cluster_sync_all();      // neither CTA exits (or frees TMEM) while its peer still runs
   if (warp == kMmaWarp) {
     __syncwarp();
     tc_fence_after_sync();
-    tmem_dealloc(tmem_base, kTmemCols);
+    if (PAIR) tmem_dealloc_pair(tmem_base, kTmemCols);
+    else tmem_dealloc(tmem_base, kTmemCols);
   }
 }
 

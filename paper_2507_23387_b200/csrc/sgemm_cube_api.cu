@@ -49,6 +49,8 @@ struct sgemm_cube_ctx {
   long long launches = 0;
   int kblock_termwise = 256;
   int kblock_elementwise = 64;
+  int cta_pair = 0;            // 1: launch the tensor-core kernels as 2-CTA clusters (cta_group::2)
+  int max_pair_clusters[3] = {0, 0, 0};   // co-resident 2-CTA clusters: <1,false>, <3,false>, <3,true>
   EncodeTiledFn encode = nullptr;
   bool attrs_set = false;
 };
@@ -87,17 +89,60 @@ int make_map(sgemm_cube_ctx* h, CUtensorMap* map, CUtensorMapDataType dt, size_t
 
 int set_kernel_attrs(sgemm_cube_ctx* h) {
   if (h->attrs_set) return SGEMM_CUBE_OK;
-  if (cudaFuncSetAttribute(sgc::tc_gemm_kernel<1, false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                           (int)sgc::TcCfg<1>::SMEM_BYTES) != cudaSuccess ||
-      cudaFuncSetAttribute(sgc::tc_gemm_kernel<3, false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                           (int)sgc::TcCfg<3>::SMEM_BYTES) != cudaSuccess ||
-      cudaFuncSetAttribute(sgc::tc_gemm_kernel<3, true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                           (int)sgc::TcCfg<3>::SMEM_BYTES) != cudaSuccess) {
+  const cudaFuncAttribute attr = cudaFuncAttributeMaxDynamicSharedMemorySize;
+  if (cudaFuncSetAttribute(sgc::tc_gemm_kernel<1, false, false>, attr, (int)sgc::TcCfg<1, false>::SMEM_BYTES) != cudaSuccess ||
+      cudaFuncSetAttribute(sgc::tc_gemm_kernel<3, false, false>, attr, (int)sgc::TcCfg<3, false>::SMEM_BYTES) != cudaSuccess ||
+      cudaFuncSetAttribute(sgc::tc_gemm_kernel<3, true, false>, attr, (int)sgc::TcCfg<3, false>::SMEM_BYTES) != cudaSuccess ||
+      cudaFuncSetAttribute(sgc::tc_gemm_kernel<1, false, true>, attr, (int)sgc::TcCfg<1, true>::SMEM_BYTES) != cudaSuccess ||
+      cudaFuncSetAttribute(sgc::tc_gemm_kernel<3, false, true>, attr, (int)sgc::TcCfg<3, true>::SMEM_BYTES) != cudaSuccess ||
+      cudaFuncSetAttribute(sgc::tc_gemm_kernel<3, true, true>, attr, (int)sgc::TcCfg<3, true>::SMEM_BYTES) != cudaSuccess) {
     cudaGetLastError();
     return SGEMM_CUBE_CUDA_ERROR;
   }
   h->attrs_set = true;
   return SGEMM_CUBE_OK;
+}
+
+// Launch one tensor-core kernel: a persistent grid of single CTAs, or of 2-CTA clusters (PAIR).
+template <int NTERMS, bool FUSED, bool PAIR>
+int launch_tc_kernel(sgemm_cube_ctx* h, int M, int N, const CUtensorMap& tmA0, const CUtensorMap& tmA1,
+                     const CUtensorMap& tmB0, const CUtensorMap& tmB1, const sgc::TcGemmParams& p,
+                     cudaStream_t st) {
+  using Cfg = sgc::TcCfg<NTERMS, PAIR>;
+  auto kernel = sgc::tc_gemm_kernel<NTERMS, FUSED, PAIR>;
+  cudaLaunchConfig_t cfg;
+  memset(&cfg, 0, sizeof(cfg));
+  cfg.blockDim = dim3(FUSED ? sgc::kFusedThreads : sgc::kTcThreads, 1, 1);
+  cfg.dynamicSmemBytes = Cfg::SMEM_BYTES;
+  cfg.stream = st;
+  cudaLaunchAttribute attrs[1];
+  const int tiles_n = (N + sgc::kBN - 1) / sgc::kBN;
+  if (PAIR) {
+    attrs[0].id = cudaLaunchAttributeClusterDimension;
+    attrs[0].val.clusterDim.x = 2;
+    attrs[0].val.clusterDim.y = 1;
+    attrs[0].val.clusterDim.z = 1;
+    cfg.attrs = attrs;
+    cfg.numAttrs = 1;
+    int& cached = h->max_pair_clusters[FUSED ? 2 : (NTERMS == 3 ? 1 : 0)];
+    if (cached == 0) {
+      cfg.gridDim = dim3(2 * h->sm_count, 1, 1);
+      int n = 0;
+      if (cudaOccupancyMaxActiveClusters(&n, kernel, &cfg) != cudaSuccess || n < 1) {
+        cudaGetLastError();
+        return SGEMM_CUBE_CUDA_ERROR;
+      }
+      cached = n;
+    }
+    const int units = ((M + 2 * sgc::kBM - 1) / (2 * sgc::kBM)) * tiles_n;
+    cfg.gridDim = dim3(2 * (units < cached ? units : cached), 1, 1);
+  } else {
+    const int units = ((M + sgc::kBM - 1) / sgc::kBM) * tiles_n;
+    cfg.gridDim = dim3(units < h->sm_count ? units : h->sm_count, 1, 1);
+  }
+  h->launches++;
+  return cudaLaunchKernelEx(&cfg, kernel, tmA0, tmA1, tmB0, tmB1, p) == cudaSuccess
+             ? SGEMM_CUBE_OK : (cudaGetLastError(), SGEMM_CUBE_CUDA_ERROR);
 }
 
 int check_gemm_dims(int M, int N, int K, int64_t lda, int64_t ldb, int64_t ldc) {
@@ -129,7 +174,7 @@ int launch_tc_gemm(sgemm_cube_ctx* h, int M, int N, int K, const uint16_t* Ahi, 
                    int64_t lda16, const uint16_t* Bhi, const uint16_t* Blo, int64_t ldb16, float* D,
                    int64_t ldd, int accumulate, int order, int kblock, float inv_scale,
                    cudaStream_t st) {
-  using Cfg = sgc::TcCfg<NTERMS>;
+  using Cfg = sgc::TcCfg<NTERMS, false>;      // BK and the A swizzle do not depend on PAIR
   int rc = set_kernel_attrs(h);
   if (rc) return rc;
   CUtensorMap tmA0, tmA1, tmB0, tmB1;
@@ -160,16 +205,13 @@ int launch_tc_gemm(sgemm_cube_ctx* h, int M, int N, int K, const uint16_t* Ahi, 
   p.inv_scale = inv_scale;
   p.err = h->err_dev;
   p.A32 = nullptr; p.lda32 = 0; p.B32 = nullptr; p.ldb32 = 0; p.scale = 1.f;
-  const int tiles = ((M + sgc::kBM - 1) / sgc::kBM) * ((N + sgc::kBN - 1) / sgc::kBN);
-  const int grid = tiles < h->sm_count ? tiles : h->sm_count;
-  sgc::tc_gemm_kernel<NTERMS, false><<<grid, sgc::kTcThreads, Cfg::SMEM_BYTES, st>>>(tmA0, tmA1, tmB0, tmB1, p);
-  h->launches++;
-  return cudaGetLastError() == cudaSuccess ? SGEMM_CUBE_OK : SGEMM_CUBE_CUDA_ERROR;
+  return h->cta_pair ? launch_tc_kernel<NTERMS, false, true>(h, M, N, tmA0, tmA1, tmB0, tmB1, p, st)
+                     : launch_tc_kernel<NTERMS, false, false>(h, M, N, tmA0, tmA1, tmB0, tmB1, p, st);
 }
 
 int launch_fused(sgemm_cube_ctx* h, int M, int N, int K, const float* A, int64_t lda, const float* B,
                  int64_t ldb, float* C, int64_t ldc, int s, int order, cudaStream_t st) {
-  using Cfg = sgc::TcCfg<3>;
+  using Cfg = sgc::TcCfg<3, false>;
   int rc = set_kernel_attrs(h);
   if (rc) return rc;
   sgc::TcGemmParams p;
@@ -187,11 +229,8 @@ int launch_fused(sgemm_cube_ctx* h, int M, int N, int K, const float* A, int64_t
   p.scale = ldexpf(1.0f, s);
   CUtensorMap unused;
   memset(&unused, 0, sizeof(unused));
-  const int tiles = ((M + sgc::kBM - 1) / sgc::kBM) * ((N + sgc::kBN - 1) / sgc::kBN);
-  const int grid = tiles < h->sm_count ? tiles : h->sm_count;
-  sgc::tc_gemm_kernel<3, true><<<grid, sgc::kFusedThreads, Cfg::SMEM_BYTES, st>>>(unused, unused, unused, unused, p);
-  h->launches++;
-  return cudaGetLastError() == cudaSuccess ? SGEMM_CUBE_OK : SGEMM_CUBE_CUDA_ERROR;
+  return h->cta_pair ? launch_tc_kernel<3, true, true>(h, M, N, unused, unused, unused, unused, p, st)
+                     : launch_tc_kernel<3, true, false>(h, M, N, unused, unused, unused, unused, p, st);
 }
 
 }  // namespace
@@ -269,6 +308,11 @@ int sgemm_cube_destroy(sgemm_cube_handle h) {
 
 int sgemm_cube_set_option(sgemm_cube_handle h, int option, int64_t value) {
   if (!h) return SGEMM_CUBE_INVALID_ARG;
+  if (option == SGEMM_CUBE_OPT_CTA_PAIR) {
+    if (value != 0 && value != 1) return SGEMM_CUBE_INVALID_ARG;
+    h->cta_pair = (int)value;
+    return SGEMM_CUBE_OK;
+  }
   if (value < 64 || value % 64 != 0 || value > (1 << 24)) return SGEMM_CUBE_INVALID_ARG;
   if (option == SGEMM_CUBE_OPT_TERMWISE_K_BLOCK) h->kblock_termwise = (int)value;
   else if (option == SGEMM_CUBE_OPT_ELEMENTWISE_K_BLOCK) h->kblock_elementwise = (int)value;

@@ -156,6 +156,8 @@ def main():
     ap.add_argument("--cpu-rows", type=int, default=2048)
     ap.add_argument("--size", type=int, default=8192,
                     help="M = N = K; values other than 8192 are for profiler captures only")
+    ap.add_argument("--strategy", default="auto", choices=["auto", "fused", "two_phase"],
+                    help="SGEMM_CUBE_OPT_STRATEGY for sgemm_cube (the bench value uses auto)")
     ap.add_argument("--entry", default="sgemm_cube", choices=["sgemm_cube", "presplit", "unfused"],
                     help="entry point timed as the step (profiler captures; the bench value is sgemm_cube)")
     ap.add_argument("--kernel-only", action="store_true",
@@ -187,6 +189,10 @@ def main():
         dist.init_process_group("nccl", device_id=torch.device(dev))
 
     h = binding.Handle(local_rank)
+    strategies = {"auto": binding.STRATEGY_AUTO, "fused": binding.STRATEGY_FUSED,
+                  "two_phase": binding.STRATEGY_TWO_PHASE}
+    h.sgemm_cube_set_option(binding.OPT_STRATEGY, strategies[args.strategy])
+    h.sgemm_cube_set_option(binding.OPT_TIME_KERNEL, 1)
     # Same seeded workload on every rank (independent replicas of the problem: weak scaling).
     A_host = torch.from_numpy(inputs.exponent_spread(0, (M, K), stream=0))
     B_host = torch.from_numpy(inputs.exponent_spread(0, (K, N), stream=1))
@@ -234,7 +240,16 @@ def main():
     st, det = h.sgemm_cube_check()
     if st != 0:
         raise SystemExit("device error %s" % hex(det))
-    per_launch_ms = [ev[i].elapsed_time(ev[i + 1]) for i in range(args.steps)]
+    # Device time of the dominant (tensor-core) kernel inside a step: events recorded by the library
+    # around that launch, read for the last timed step and for a few more steps of the same call.
+    kernel_samples = []
+    if args.entry == "sgemm_cube":
+        kernel_samples.append(h.sgemm_cube_last_kernel_ms())
+        for _ in range(5):
+            step()
+            kernel_samples.append(h.sgemm_cube_last_kernel_ms())
+    else:
+        kernel_samples = [ev[i].elapsed_time(ev[i + 1]) for i in range(args.steps)]
     t = torch.tensor([total_ms], device=dev, dtype=torch.float64)
     if world > 1:
         dist.all_reduce(t, op=dist.ReduceOp.MAX)
@@ -264,9 +279,13 @@ def main():
         t_pre = timed(lambda: h.sgemm_cube_presplit(Ahi, Alo, Bhi, Blo, C, SCALE_EXP, binding.TERMWISE))
         t_unf = timed(lambda: h.sgemm_cube_unfused(A, B, C, SCALE_EXP, binding.TERMWISE))
         t_ele = timed(lambda: h.sgemm_cube(A, B, C, SCALE_EXP, binding.ELEMENTWISE))
-        extra = {"presplit_kernel_tflops": flops / t_pre / 1e9,
+        h.sgemm_cube_set_option(binding.OPT_STRATEGY, binding.STRATEGY_FUSED)
+        t_fus = timed(lambda: h.sgemm_cube(A, B, C, SCALE_EXP, binding.TERMWISE))
+        h.sgemm_cube_set_option(binding.OPT_STRATEGY, strategies[args.strategy])
+        extra = {"three_product_kernel_alone_tflops": flops / t_pre / 1e9,
                  "unfused_split_3gemm_tflops": flops / t_unf / 1e9,
-                 "fused_elementwise_tflops": flops / t_ele / 1e9,
+                 "elementwise_order_tflops": flops / t_ele / 1e9,
+                 "fused_converter_kernel_tflops": flops / t_fus / 1e9,
                  "split_kernel_gbs": 8.0 * M * K / t_split / 1e6}
         del Ahi, Alo, Bhi, Blo
 
@@ -298,7 +317,7 @@ def main():
 
     if rank == 0:
         peaks = measured_peaks()
-        kernel_ms = statistics.mean(per_launch_ms)
+        kernel_ms = statistics.mean(kernel_samples)
         achieved = 3.0 * flops / (kernel_ms * 1e-3) / 1e12      # FP16 tensor-core TFLOP/s
         peak = peaks["bf16_tflops"]
         sm_count = torch.cuda.get_device_properties(local_rank).multi_processor_count
@@ -310,7 +329,9 @@ def main():
             "warmup": warmup, "ms_per_step": ms_per_step, "higher_is_better": True,
             "scaling": "weak", "vs_baseline": None, "dtype": "f16 products, f32 accumulate",
             "data": "synthetic",
-            "config": {"workload": WORKLOAD, "entry_point": "sgemm_cube (fused kernel)",
+            "config": {"workload": WORKLOAD, "entry_point": "sgemm_cube, strategy %s: split kernel x2 + three-product "
+                                      "tensor-core kernel per step" % args.strategy
+                       if args.strategy != "fused" else "sgemm_cube, strategy fused: one kernel per step",
                        "l2": "inputs (512 MiB) larger than L2; no flush",
                        "parallelism": "replicas x%d" % world if world > 1 else "1 GPU"},
             "clocks": clocks,

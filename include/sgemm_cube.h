@@ -67,8 +67,28 @@ enum {
   SGEMM_CUBE_OPT_ELEMENTWISE_K_BLOCK = 1,
   /* 1: run the tensor-core kernels as clusters of two CTAs that share one
    * tcgen05.mma.cta_group::2 (256 x 256 tile per pair, each CTA loading half of the B tile);
-   * 0: one CTA per 128 x 256 tile.  Same arithmetic either way. */
-  SGEMM_CUBE_OPT_CTA_PAIR = 2
+   * 0: one CTA per 128 x 256 tile; 2 (default): pairs when the problem has at least four waves of
+   * pair tiles.  Same arithmetic, bit-identical results either way. */
+  SGEMM_CUBE_OPT_CTA_PAIR = 2,
+  /* How sgemm_cube computes (same arithmetic and bracketing, bit-identical results):
+   * SGEMM_CUBE_STRATEGY_FUSED     one kernel; converter warps split FP32 tiles on the fly, no FP16
+   *                               copy of A or B exists in device memory, no workspace;
+   * SGEMM_CUBE_STRATEGY_TWO_PHASE the split kernel writes the FP16 words of A and B once into the
+   *                               handle's workspace (4 bytes per element of A and B, grown with
+   *                               cudaMalloc on first use), then one kernel forms all three
+   *                               products and the reconstruction;
+   * SGEMM_CUBE_STRATEGY_AUTO      (default) TWO_PHASE when M*N*K >= 2^30 and the workspace can be
+   *                               had, FUSED otherwise. */
+  SGEMM_CUBE_OPT_STRATEGY = 3,
+  /* 1: sgemm_cube records CUDA events around its tensor-core kernel, for
+   * sgemm_cube_last_kernel_ms.  Default 0. */
+  SGEMM_CUBE_OPT_TIME_KERNEL = 4
+};
+
+enum {
+  SGEMM_CUBE_STRATEGY_AUTO = 0,
+  SGEMM_CUBE_STRATEGY_FUSED = 1,
+  SGEMM_CUBE_STRATEGY_TWO_PHASE = 2
 };
 
 /* Create a handle bound to CUDA device `device`.  Allocates a small device error word; the
@@ -98,17 +118,21 @@ int sgemm_cube_split(sgemm_cube_handle h, int rows, int cols,
                      uint16_t* hi_dev, uint16_t* lo_dev, int64_t ldh,
                      int scale_exp, void* stream);
 
-/* Fused SGEMM-cube (paper Eq. recover_eqn with Eq. termwise or Eq. elementwise):
- *   C = hi_A hi_B + 2^-s (lo_A hi_B + hi_A lo_B),   hi/lo produced on the fly inside the kernel
- * (no FP16 copy of A or B goes through device memory), FP16 x FP16 products on the tensor cores
- * with FP32 accumulation, C overwritten (no alpha/beta).
+/* SGEMM-cube (paper Eq. recover_eqn with Eq. termwise or Eq. elementwise):
+ *   C = hi_A hi_B + 2^-s (lo_A hi_B + hi_A lo_B),
+ * hi = fl16(x), lo = fl16((x - hi) 2^s) as in sgemm_cube_split, FP16 x FP16 products on the tensor
+ * cores with FP32 accumulation, the reconstruction in FP32; C overwritten (no alpha/beta).
+ * The operand split runs either inside the product kernel (converter warps, no FP16 copy of A or
+ * B in device memory) or once up front into the handle's workspace: see SGEMM_CUBE_OPT_STRATEGY.
+ * Both give bit-identical C.
  *   A_dev  M x K FP32, lda >= K     (device, read)
  *   B_dev  K x N FP32, ldb >= N     (device, read)
  *   C_dev  M x N FP32, ldc >= N     (device, written)
  *   scale_exp s in [0, 24]; accumulation_order SGEMM_CUBE_TERMWISE or SGEMM_CUBE_ELEMENTWISE
  * Alignment: A_dev, B_dev 16-byte aligned and lda % 4 == 0, ldb % 4 == 0 (else MISALIGNED).
  * C_dev may have any alignment.  M, N, K >= 1, any values (ragged edges are handled).
- * Errors: INVALID_ARG, MISALIGNED, CUDA_ERROR. */
+ * Errors: INVALID_ARG, MISALIGNED, CUDA_ERROR (ALLOC_FAILED only with the TWO_PHASE strategy
+ * forced; AUTO falls back to the fused kernel when the workspace cannot be had). */
 int sgemm_cube(sgemm_cube_handle h, int M, int N, int K,
                const float* A_dev, int64_t lda,
                const float* B_dev, int64_t ldb,
@@ -204,6 +228,11 @@ int sgemm_cube_check(sgemm_cube_handle h, void* stream, uint32_t* detail_out);
 
 /* Number of kernels this handle has launched since creation (for launch accounting). */
 int64_t sgemm_cube_launch_count(sgemm_cube_handle h);
+
+/* Device time, in milliseconds, of the tensor-core kernel of the most recent sgemm_cube call
+ * (requires SGEMM_CUBE_OPT_TIME_KERNEL = 1 before that call; waits for the kernel to finish).
+ * Errors: INVALID_ARG (timing off, or no call yet), CUDA_ERROR. */
+int sgemm_cube_last_kernel_ms(sgemm_cube_handle h, float* ms_out);
 
 /* Text for a status code (static storage; never NULL). */
 const char* sgemm_cube_status_string(int status);

@@ -15,11 +15,12 @@ LIB_PATH = os.path.join(HERE, "libsgemm_cube.so")
 OK, INVALID_ARG, MISALIGNED, CUDA_ERROR, DEVICE_TIMEOUT, UNSUPPORTED_ARCH, ALLOC_FAILED, TOO_LARGE = range(8)
 STATIC_SCRATCH_BYTES = 32 << 20
 TERMWISE, ELEMENTWISE = 0, 1
-OPT_TERMWISE_K_BLOCK, OPT_ELEMENTWISE_K_BLOCK, OPT_CTA_PAIR = 0, 1, 2
+OPT_TERMWISE_K_BLOCK, OPT_ELEMENTWISE_K_BLOCK, OPT_CTA_PAIR, OPT_STRATEGY, OPT_TIME_KERNEL = range(5)
+STRATEGY_AUTO, STRATEGY_FUSED, STRATEGY_TWO_PHASE = 0, 1, 2
 
 EXPORTS = ["sgemm_cube_create", "sgemm_cube_destroy", "sgemm_cube_set_option", "sgemm_cube_split",
            "sgemm_cube", "sgemm_cube_unfused", "sgemm_cube_presplit", "sgemm_cube_hgemm",
-           "sgemm_cube_host", "sgemm_cube_unfused_static", "sgemm_cube_check", "sgemm_cube_launch_count",
+           "sgemm_cube_host", "sgemm_cube_unfused_static", "sgemm_cube_check", "sgemm_cube_launch_count", "sgemm_cube_last_kernel_ms",
            "sgemm_cube_status_string", "sgemm_cube_version"]
 
 _lib = None
@@ -54,6 +55,7 @@ def load():
     lib.sgemm_cube_hgemm.argtypes = [vp, i32, i32, i32, vp, i64, vp, i64, vp, i64, i32, vp]
     lib.sgemm_cube_unfused_static.argtypes = [i32, i32, i32, vp, i64, vp, i64, vp, i64, i32, vp]
     lib.sgemm_cube_check.argtypes = [vp, vp, ctypes.POINTER(ctypes.c_uint32)]
+    lib.sgemm_cube_last_kernel_ms.argtypes = [vp, ctypes.POINTER(ctypes.c_float)]
     lib.sgemm_cube_launch_count.argtypes = [vp]
     lib.sgemm_cube_launch_count.restype = i64
     lib.sgemm_cube_status_string.argtypes = [i32]
@@ -190,3 +192,8 @@ class Handle:
 
     def sgemm_cube_launch_count(self) -> int:
         return int(load().sgemm_cube_launch_count(self._h))
+
+    def sgemm_cube_last_kernel_ms(self) -> float:
+        ms = ctypes.c_float(0.0)
+        _check(load().sgemm_cube_last_kernel_ms(self._h, ctypes.byref(ms)), "sgemm_cube_last_kernel_ms")
+        return float(ms.value)

@@ -12,7 +12,7 @@
 // Structure (one persistent CTA per SM):
 //   warps 0-7    accumulate/epilogue warps: tcgen05.ld the TMEM partial sums, add them with FP32
 //                round-to-nearest into running sums held in registers, form C, store it
-//   not FUSED (320 threads): warp 8 = TMA producer (FP16 tiles global -> shared, swizzled UMMA
+//   not FUSED (384 threads): warp 8 = TMA producer (FP16 tiles global -> shared, swizzled UMMA
 //                layout), warp 9 = MMA issuer
 //   FUSED (512 threads): warps 8-14 = converter warps: FP32 tiles global -> registers -> (hi, lo)
 //                FP16 words -> shared memory, written directly in the swizzled UMMA layout;
@@ -44,7 +44,7 @@ namespace sgc {
 constexpr int kBM = 128;            // CTA tile rows  (UMMA M)
 constexpr int kBN = 256;            // CTA tile cols  (UMMA N)
 constexpr int kNumEpiWarps = 8;     // warps 0-7
-constexpr int kTcThreads = 320;     // not FUSED: + TMA warp + MMA warp
+constexpr int kTcThreads = 384;     // not FUSED: + TMA warp + MMA warp (+ 2 idle warps: whole warpgroup)
 constexpr int kFusedThreads = 512;  // FUSED: + 7 converter warps + MMA warp
 constexpr int kNumConvWarps = 7;
 constexpr int kConvThreads = kNumConvWarps * 32;   // 224
@@ -97,7 +97,9 @@ struct TcCfg {
   static constexpr uint32_t B_TILE = BK * BN_CTA * 2;     // one FP16 B tile (this CTA's columns)
   static constexpr uint32_t STAGE_BYTES = (NTERMS == 1) ? (A_TILE + B_TILE) : 2 * (A_TILE + B_TILE);
   static constexpr int STAGES = (196608 / STAGE_BYTES) > 8 ? 8 : (196608 / STAGE_BYTES);
-  static constexpr uint32_t SMEM_BYTES = STAGES * STAGE_BYTES + 1024 /*align*/ + 256 /*barriers*/;
+  static constexpr uint32_t STORE_STAGING = kNumEpiWarps * 4096;   // 32 rows x 128 bytes per warp
+  static constexpr uint32_t SMEM_BYTES =
+      STAGES * STAGE_BYTES + 1024 /*align*/ + 256 /*barriers*/ + STORE_STAGING;
 };
 
 // Tile rasterisation: groups of 8 tile-rows are walked column by column so that the CTAs
@@ -260,6 +262,7 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA0, const __grid_constant__
   uint64_t* drain_bar = bars + 2 * STAGES + 4;   // [1]
   uint32_t* tmem_base_slot = reinterpret_cast<uint32_t*>(bars + 2 * STAGES + 5);
   volatile uint32_t* abort_flag = tmem_base_slot + 1;
+  uint8_t* store_staging = smem + STAGES * Cfg::STAGE_BYTES + 256;   // epilogue transposition buffers
 
   const int warp = threadIdx.x >> 5;
   const int lane = threadIdx.x & 31;
@@ -319,6 +322,7 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA0, const __grid_constant__
   // that the code below it is compiled against the new limit.
   if (warp < kNumEpiWarps) {
     if (FUSED) setmaxnreg_inc<168>();
+    else setmaxnreg_inc<208>();       // 384 threads x 168: 256 x 208 + 128 x 56 fits the pool
     // ------------------------------------------------------------------ accumulate / epilogue
     const int quarter = warp & 3;                 // TMEM lanes 32*quarter .. +31 (warp id mod 4)
     const int half = warp >> 2;                   // columns [128*half, 128*half + 128)
@@ -412,14 +416,63 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA0, const __grid_constant__
         if (lane == 0) arrive_tempty(1);
         drains[1]++;
       }
+      if (vec_ok) {
+        // Each thread owns one row of the tile; storing straight from registers would write 16
+        // bytes per row per instruction.  Instead 32 x 32 blocks go through a per-warp staging
+        // buffer (16-byte chunks XOR-swizzled by row: conflict-free both ways) and leave as
+        // 128-byte row segments, four rows per store instruction.
+        const uint32_t stg = smem_u32(store_staging + warp * 4096);
+        const int row0 = tm * kBM + quarter * 32;
 #pragma unroll
-      for (int g = 0; g < 8; ++g)
-        store16(p.D, p.ldd, p.M, p.N, row, col_base + g * 16, &S[g * 16], vec_ok,
-                (NTERMS == 1) ? p.accumulate : 0);
+        for (int g = 0; g < 4; ++g) {
+#pragma unroll
+          for (int q = 0; q < 8; ++q)
+            asm volatile("st.shared.v4.f32 [%0], {%1, %2, %3, %4};" ::"r"(
+                             stg + lane * 128 + ((q ^ (lane & 7)) << 4)),
+                         "f"(S[g * 32 + 4 * q]), "f"(S[g * 32 + 4 * q + 1]), "f"(S[g * 32 + 4 * q + 2]),
+                         "f"(S[g * 32 + 4 * q + 3])
+                         : "memory");
+          __syncwarp();
+          const int q = lane & 7;
+          const int col = col_base + g * 32 + q * 4;
+#pragma unroll
+          for (int i = 0; i < 8; ++i) {
+            const int r = i * 4 + (lane >> 3);
+            float4 v;
+            asm volatile("ld.shared.v4.f32 {%0, %1, %2, %3}, [%4];"
+                         : "=f"(v.x), "=f"(v.y), "=f"(v.z), "=f"(v.w)
+                         : "r"(stg + r * 128 + ((q ^ (r & 7)) << 4))
+                         : "memory");
+            const int grow = row0 + r;
+            if (grow < p.M && col < p.N) {
+              float* dst = p.D + (long long)grow * p.ldd + col;
+              if (col + 4 <= p.N) {
+                if (NTERMS == 1 && p.accumulate) {
+                  const float4 old = *reinterpret_cast<const float4*>(dst);
+                  v.x = __fadd_rn(old.x, v.x); v.y = __fadd_rn(old.y, v.y);
+                  v.z = __fadd_rn(old.z, v.z); v.w = __fadd_rn(old.w, v.w);
+                }
+                *reinterpret_cast<float4*>(dst) = v;
+              } else {
+                const float e[4] = {v.x, v.y, v.z, v.w};
+                for (int j = 0; j < 4 && col + j < p.N; ++j)
+                  dst[j] = (NTERMS == 1 && p.accumulate) ? __fadd_rn(dst[j], e[j]) : e[j];
+              }
+            }
+          }
+          __syncwarp();
+        }
+      } else {
+#pragma unroll
+        for (int g = 0; g < 8; ++g)
+          store16(p.D, p.ldd, p.M, p.N, row, col_base + g * 16, &S[g * 16], false,
+                  (NTERMS == 1) ? p.accumulate : 0);
+      }
       SGC_TADD(8, blockIdx.x == 0 && threadIdx.x == 0);
     }
   } else if (warp == kMmaWarp) {
     if (FUSED) setmaxnreg_dec<88>();
+    else setmaxnreg_dec<56>();
     // ------------------------------------------------------------------ MMA issuer
     if (lane == 0 && leader) {
       constexpr uint32_t idesc =
@@ -544,8 +597,9 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA0, const __grid_constant__
       mbar_wait_bounded(drain_bar, 0, nullptr, p.err, kErrDrainWait);
     }
   } else if (!FUSED) {
+    setmaxnreg_dec<56>();
     // ------------------------------------------------------------------ TMA producer (warp 8)
-    if (lane == 0) {
+    if (warp == kProducerWarp && lane == 0) {
       uint32_t it = 0;
       bool ok = true;
       auto load = [&](void* dst, const CUtensorMap* map, int x, int y, uint64_t* bar) {

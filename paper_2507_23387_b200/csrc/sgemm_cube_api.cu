@@ -49,7 +49,11 @@ struct sgemm_cube_ctx {
   long long launches = 0;
   int kblock_termwise = 256;
   int kblock_elementwise = 64;
-  int cta_pair = 0;            // 1: launch the tensor-core kernels as 2-CTA clusters (cta_group::2)
+  int cta_pair = 0;            // 0/1: never/always 2-CTA clusters (cta_group::2); 2: by problem size
+  int strategy = 0;            // sgemm_cube: 0 auto, 1 fused kernel, 2 split kernel + 3-product kernel
+  int time_kernel = 0;         // record events around the tensor-core kernel of sgemm_cube
+  cudaEvent_t ev0 = nullptr, ev1 = nullptr;
+  bool ev_recorded = false;
   int max_pair_clusters[3] = {0, 0, 0};   // co-resident 2-CTA clusters: <1,false>, <3,false>, <3,true>
   EncodeTiledFn encode = nullptr;
   bool attrs_set = false;
@@ -101,6 +105,14 @@ int set_kernel_attrs(sgemm_cube_ctx* h) {
   }
   h->attrs_set = true;
   return SGEMM_CUBE_OK;
+}
+
+// 2-CTA clusters pay off once there are enough 256 x 256 pair tiles to keep every SM pair busy
+// for several waves; below that the finer 128 x 256 tiles balance better.
+bool use_pair(const sgemm_cube_ctx* h, int M, int N) {
+  if (h->cta_pair != 2) return h->cta_pair == 1;
+  const long long pair_tiles = (long long)((M + 255) / 256) * ((N + 255) / 256);
+  return pair_tiles >= 4LL * (h->sm_count / 2);
 }
 
 // Launch one tensor-core kernel: a persistent grid of single CTAs, or of 2-CTA clusters (PAIR).
@@ -205,8 +217,8 @@ int launch_tc_gemm(sgemm_cube_ctx* h, int M, int N, int K, const uint16_t* Ahi, 
   p.inv_scale = inv_scale;
   p.err = h->err_dev;
   p.A32 = nullptr; p.lda32 = 0; p.B32 = nullptr; p.ldb32 = 0; p.scale = 1.f;
-  return h->cta_pair ? launch_tc_kernel<NTERMS, false, true>(h, M, N, tmA0, tmA1, tmB0, tmB1, p, st)
-                     : launch_tc_kernel<NTERMS, false, false>(h, M, N, tmA0, tmA1, tmB0, tmB1, p, st);
+  return use_pair(h, M, N) ? launch_tc_kernel<NTERMS, false, true>(h, M, N, tmA0, tmA1, tmB0, tmB1, p, st)
+                           : launch_tc_kernel<NTERMS, false, false>(h, M, N, tmA0, tmA1, tmB0, tmB1, p, st);
 }
 
 int launch_fused(sgemm_cube_ctx* h, int M, int N, int K, const float* A, int64_t lda, const float* B,
@@ -229,8 +241,50 @@ int launch_fused(sgemm_cube_ctx* h, int M, int N, int K, const float* A, int64_t
   p.scale = ldexpf(1.0f, s);
   CUtensorMap unused;
   memset(&unused, 0, sizeof(unused));
-  return h->cta_pair ? launch_tc_kernel<3, true, true>(h, M, N, unused, unused, unused, unused, p, st)
-                     : launch_tc_kernel<3, true, false>(h, M, N, unused, unused, unused, unused, p, st);
+  return use_pair(h, M, N) ? launch_tc_kernel<3, true, true>(h, M, N, unused, unused, unused, unused, p, st)
+                           : launch_tc_kernel<3, true, false>(h, M, N, unused, unused, unused, unused, p, st);
+}
+
+// sgemm_cube, strategy "two-phase": split both operands once into the handle's workspace, then one
+// three-product kernel on the FP16 words.  Same arithmetic and bracketing as the fused kernel.
+int launch_two_phase(sgemm_cube_ctx* h, int M, int N, int K, const float* A, int64_t lda, const float* B,
+                     int64_t ldb, float* C, int64_t ldc, int s, int order, cudaStream_t st) {
+  const size_t ldA16 = round_up((size_t)K, 8), ldB16 = round_up((size_t)N, 8);
+  const size_t szA = round_up((size_t)M * ldA16 * 2, 256), szB = round_up((size_t)K * ldB16 * 2, 256);
+  int rc = grow(&h->ws, &h->ws_bytes, 2 * szA + 2 * szB);
+  if (rc) return rc;
+  uint8_t* w = static_cast<uint8_t*>(h->ws);
+  uint16_t* Ahi = reinterpret_cast<uint16_t*>(w);
+  uint16_t* Alo = reinterpret_cast<uint16_t*>(w + szA);
+  uint16_t* Bhi = reinterpret_cast<uint16_t*>(w + 2 * szA);
+  uint16_t* Blo = reinterpret_cast<uint16_t*>(w + 2 * szA + szB);
+  if ((rc = launch_split(h, M, K, A, lda, Ahi, Alo, (int64_t)ldA16, s, st))) return rc;
+  if ((rc = launch_split(h, K, N, B, ldb, Bhi, Blo, (int64_t)ldB16, s, st))) return rc;
+  const int kblock = (order == SGEMM_CUBE_TERMWISE) ? h->kblock_termwise : h->kblock_elementwise;
+  if (h->time_kernel && h->ev0) cudaEventRecord(h->ev0, st);
+  rc = launch_tc_gemm<3>(h, M, N, K, Ahi, Alo, (int64_t)ldA16, Bhi, Blo, (int64_t)ldB16, C, ldc, 0, order,
+                         kblock, ldexpf(1.0f, -s), st);
+  if (h->time_kernel && h->ev1) { cudaEventRecord(h->ev1, st); h->ev_recorded = true; }
+  return rc;
+}
+
+// The entry point's strategy choice.  The fused kernel re-splits every operand tile once per
+// output tile and has to pull FP32 tiles (twice the bytes of the FP16 words) through L2 for each
+// of them, which bounds it well below the tensor-core rate on large problems; there the split is
+// done once up front.  Small problems keep the single launch.
+int launch_sgemm_cube(sgemm_cube_ctx* h, int M, int N, int K, const float* A, int64_t lda, const float* B,
+                      int64_t ldb, float* C, int64_t ldc, int s, int order, cudaStream_t st) {
+  bool two_phase = (h->strategy == 2) ||
+                   (h->strategy == 0 && (double)M * (double)N * (double)K >= 1024.0 * 1024.0 * 1024.0);
+  if (two_phase) {
+    int rc = launch_two_phase(h, M, N, K, A, lda, B, ldb, C, ldc, s, order, st);
+    if (rc != SGEMM_CUBE_ALLOC_FAILED || h->strategy == 2) return rc;
+    // no room for the FP16 words: the fused kernel needs no workspace
+  }
+  if (h->time_kernel && h->ev0) cudaEventRecord(h->ev0, st);
+  int rc = launch_fused(h, M, N, K, A, lda, B, ldb, C, ldc, s, order, st);
+  if (h->time_kernel && h->ev1) { cudaEventRecord(h->ev1, st); h->ev_recorded = true; }
+  return rc;
 }
 
 }  // namespace
@@ -301,6 +355,8 @@ int sgemm_cube_destroy(sgemm_cube_handle h) {
     rc = SGEMM_CUBE_DEVICE_TIMEOUT;
   if (h->ws) cudaFree(h->ws);
   if (h->host_ws) cudaFree(h->host_ws);
+  if (h->ev0) cudaEventDestroy(h->ev0);
+  if (h->ev1) cudaEventDestroy(h->ev1);
   cudaFree(h->err_dev);
   delete h;
   return rc;
@@ -309,8 +365,26 @@ int sgemm_cube_destroy(sgemm_cube_handle h) {
 int sgemm_cube_set_option(sgemm_cube_handle h, int option, int64_t value) {
   if (!h) return SGEMM_CUBE_INVALID_ARG;
   if (option == SGEMM_CUBE_OPT_CTA_PAIR) {
-    if (value != 0 && value != 1) return SGEMM_CUBE_INVALID_ARG;
+    if (value < 0 || value > 2) return SGEMM_CUBE_INVALID_ARG;
     h->cta_pair = (int)value;
+    return SGEMM_CUBE_OK;
+  }
+  if (option == SGEMM_CUBE_OPT_STRATEGY) {
+    if (value < 0 || value > 2) return SGEMM_CUBE_INVALID_ARG;
+    h->strategy = (int)value;
+    return SGEMM_CUBE_OK;
+  }
+  if (option == SGEMM_CUBE_OPT_TIME_KERNEL) {
+    if (value != 0 && value != 1) return SGEMM_CUBE_INVALID_ARG;
+    DeviceGuard g(h->device);
+    if (value && !h->ev0) {
+      if (cudaEventCreate(&h->ev0) != cudaSuccess || cudaEventCreate(&h->ev1) != cudaSuccess) {
+        cudaGetLastError();
+        return SGEMM_CUBE_CUDA_ERROR;
+      }
+    }
+    h->time_kernel = (int)value;
+    h->ev_recorded = false;
     return SGEMM_CUBE_OK;
   }
   if (value < 64 || value % 64 != 0 || value > (1 << 24)) return SGEMM_CUBE_INVALID_ARG;
@@ -340,8 +414,8 @@ int sgemm_cube(sgemm_cube_handle h, int M, int N, int K, const float* A, int64_t
   if (!aligned16(A) || !aligned16(B) || (lda % 4) || (ldb % 4)) return SGEMM_CUBE_MISALIGNED;
   DeviceGuard g(h->device);
   if (!g.ok) return SGEMM_CUBE_CUDA_ERROR;
-  return launch_fused(h, M, N, K, A, lda, B, ldb, C, ldc, scale_exp, order,
-                      static_cast<cudaStream_t>(stream));
+  return launch_sgemm_cube(h, M, N, K, A, lda, B, ldb, C, ldc, scale_exp, order,
+                           static_cast<cudaStream_t>(stream));
 }
 
 int sgemm_cube_presplit(sgemm_cube_handle h, int M, int N, int K, const uint16_t* Ahi,
@@ -442,7 +516,7 @@ int sgemm_cube_host(sgemm_cube_handle h, int M, int N, int K, const float* A_hos
     cudaGetLastError();
     return SGEMM_CUBE_CUDA_ERROR;
   }
-  rc = launch_fused(h, M, N, K, dA, (int64_t)ldA, dB, (int64_t)ldB, dC, (int64_t)ldC, scale_exp, order, st);
+  rc = launch_sgemm_cube(h, M, N, K, dA, (int64_t)ldA, dB, (int64_t)ldB, dC, (int64_t)ldC, scale_exp, order, st);
   if (rc) return rc;
   if (cudaMemcpy2DAsync(C_host, (size_t)ldc * 4, dC, ldC * 4, (size_t)N * 4, M, cudaMemcpyDeviceToHost, st) != cudaSuccess) {
     cudaGetLastError();
@@ -471,6 +545,17 @@ int sgemm_cube_check(sgemm_cube_handle h, void* stream, uint32_t* detail_out) {
 }
 
 int64_t sgemm_cube_launch_count(sgemm_cube_handle h) { return h ? h->launches : -1; }
+
+int sgemm_cube_last_kernel_ms(sgemm_cube_handle h, float* ms_out) {
+  if (!h || !ms_out || !h->time_kernel || !h->ev_recorded) return SGEMM_CUBE_INVALID_ARG;
+  DeviceGuard g(h->device);
+  if (cudaEventSynchronize(h->ev1) != cudaSuccess ||
+      cudaEventElapsedTime(ms_out, h->ev0, h->ev1) != cudaSuccess) {
+    cudaGetLastError();
+    return SGEMM_CUBE_CUDA_ERROR;
+  }
+  return SGEMM_CUBE_OK;
+}
 
 }  // extern "C"
 

@@ -31,8 +31,12 @@ def run(h, path, Ad, Bd, s, order):
     """Run one entry point on device operands; returns C as numpy."""
     M, N = Ad.shape[0], Bd.shape[1]
     C = torch.full((M, N), float("nan"), device="cuda:0")
-    if path == "fused":
-        h.sgemm_cube(Ad, Bd, C, s, order)
+    if path in STRATEGY:
+        h.sgemm_cube_set_option(binding.OPT_STRATEGY, STRATEGY[path])
+        try:
+            h.sgemm_cube(Ad, Bd, C, s, order)
+        finally:
+            h.sgemm_cube_set_option(binding.OPT_STRATEGY, binding.STRATEGY_AUTO)
     elif path == "unfused":
         h.sgemm_cube_unfused(Ad, Bd, C, s, order)
     elif path == "presplit":
@@ -49,7 +53,12 @@ def run(h, path, Ad, Bd, s, order):
     return C.cpu().numpy()
 
 
-PATHS = [("fused", T), ("fused", E), ("presplit", T), ("presplit", E), ("unfused", T)]
+# sgemm_cube with each strategy forced ("fused": converter warps; "two_phase": split kernel + one
+# three-product kernel; "auto": the library's choice), and the other entry points.
+STRATEGY = {"fused": binding.STRATEGY_FUSED, "two_phase": binding.STRATEGY_TWO_PHASE,
+            "auto": binding.STRATEGY_AUTO}
+PATHS = [("fused", T), ("fused", E), ("two_phase", T), ("two_phase", E), ("presplit", T),
+         ("presplit", E), ("unfused", T)]
 
 
 @pytest.mark.parametrize("path,order", PATHS)
@@ -122,14 +131,33 @@ def test_output_leading_dimension_and_alignment(handle, path, order):
     assert torch.all(big[:, :3] == -7.0) and torch.all(big[:, 3 + N:] == -7.0)
 
 
-def test_fused_and_presplit_agree_bitwise(handle):
+def test_strategies_agree_bitwise(handle):
     # Same products, same accumulation structure: the on-the-fly split must reproduce the words of
-    # the split kernel exactly, so the two results are identical.
+    # the split kernel exactly, so all strategies give identical results.
     A, B = inputs.make_pair("exponent_spread", 4, 384, 512, 640)
     for order in (T, E):
         C1 = run(handle, "fused", to_dev(A), to_dev(B), 11, order)
         C2 = run(handle, "presplit", to_dev(A), to_dev(B), 11, order)
-        assert np.array_equal(C1, C2)
+        C3 = run(handle, "two_phase", to_dev(A), to_dev(B), 11, order)
+        assert np.array_equal(C1, C2) and np.array_equal(C1, C3)
+
+
+@pytest.mark.parametrize("path,order", PATHS)
+def test_cta_pair_mode_is_bit_identical(handle, path, order):
+    # tcgen05.mma.cta_group::2 (two CTAs per 256 x 256 tile) against one CTA per 128 x 256 tile.
+    res = {}
+    try:
+        for pair in (0, 1):
+            handle.sgemm_cube_set_option(binding.OPT_CTA_PAIR, pair)
+            res[pair] = [run(handle, path, padded_dev(A, 4), padded_dev(B, 4), 11, order)
+                         for (A, B) in (inputs.make_pair("normal", 6, M, N, K)
+                                        for (M, N, K) in [(512, 768, 520), (129, 300, 97), (1024, 256, 2048)])]
+    finally:
+        handle.sgemm_cube_set_option(binding.OPT_CTA_PAIR, 2)
+    for a, b in zip(res[0], res[1]):
+        assert np.array_equal(a, b)
+    A, B = inputs.make_pair("normal", 6, 129, 300, 97)
+    gates(res[1][1], A, B, 11, order, label="pair %s" % path)
 
 
 def test_k_block_option_changes_bracketing_not_validity(handle):
@@ -158,11 +186,7 @@ def test_config2_4096_cubed_sampled_rows(handle, path, order):
     rows = np.sort(np.random.default_rng(0).choice(n, 48, replace=False))
     Ad, Bd = to_dev(A), to_dev(B)
     C = torch.empty((n, n), device="cuda:0")
-    getattr(handle, "sgemm_cube" if path == "fused" else "sgemm_cube_unfused")(Ad, Bd, C, 11, order) \
-        if path != "presplit" else None
-    if path == "presplit":
-        C = torch.from_numpy(run(handle, path, Ad, Bd, 11, order)).to("cuda:0")
-    assert handle.sgemm_cube_check()[0] == 0
+    C = torch.from_numpy(run(handle, path, Ad, Bd, 11, order)).to("cuda:0")
     _sampled_rows_check(handle, path, order, A[rows], B, C, rows, "4096^3 %s %d" % (path, order))
 
 
@@ -184,7 +208,7 @@ def test_config2_orders_compared(handle):
     assert 0.25 < errs[T] / errs[E] < 4.0
 
 
-@pytest.mark.parametrize("path,order", [("fused", T), ("presplit", T), ("unfused", T)])
+@pytest.mark.parametrize("path,order", [("auto", T), ("fused", T), ("presplit", T), ("unfused", T)])
 def test_config3_8192_cubed_exponent_spread_sampled_rows(handle, path, order):
     n = 8192
     A, B = inputs.make_pair("exponent_spread", 0, n, n, n)
@@ -194,7 +218,8 @@ def test_config3_8192_cubed_exponent_spread_sampled_rows(handle, path, order):
     gates(C[torch.as_tensor(rows)].numpy(), A[rows], B, 11, order, label="8192^3 %s" % path)
 
 
-@pytest.mark.parametrize("path,order", [("fused", T), ("fused", E), ("presplit", T), ("unfused", T)])
+@pytest.mark.parametrize("path,order", [("auto", T), ("auto", E), ("fused", T), ("fused", E),
+                                        ("presplit", T), ("unfused", T)])
 def test_config4_long_k_normal(handle, path, order):
     M = N = 1024
     K = 65536
@@ -275,6 +300,8 @@ def test_argument_errors(handle):
     assert call(A=None) == binding.INVALID_ARG
     assert call(A=p(A) + 4) == binding.MISALIGNED
     assert call(lda=18) == binding.MISALIGNED
+    for opt, bad in ((binding.OPT_STRATEGY, 3), (binding.OPT_CTA_PAIR, 3), (binding.OPT_TIME_KERNEL, 2), (9, 0)):
+        assert lib.sgemm_cube_set_option(handle._h, opt, bad) == binding.INVALID_ARG
     assert lib.sgemm_cube_unfused(handle._h, 8, 8, 16, p(A), 16, p(B), 8, p(C), 8, 11, 1,
                                   None) == binding.INVALID_ARG       # unfused is termwise only
     assert handle.sgemm_cube_check()[0] == 0

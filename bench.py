@@ -33,9 +33,10 @@ WORKLOAD = "M=N=K=8192 FP32 GEMM, entries (+/-)u*2^e, u~U[1,2), e~U{-10..10}, s=
 METRIC = "FP32-equiv TFLOP/s (2MNK/t) at 8192^3"
 UNIT = "TFLOP/s"
 
-# DRAM traffic of one launch of the fused kernel at this workload, from the ncu capture summarised
-# in profiles/ (dram__bytes_read.sum + dram__bytes_write.sum); None until a capture exists.
-FUSED_KERNEL_DRAM_BYTES_PER_LAUNCH = None
+# DRAM traffic of one launch of the dominant kernel (the three-product tensor-core kernel) at this
+# workload: dram__bytes_read.sum + dram__bytes_write.sum of the full-size one-pass ncu capture
+# summarised in profiles/three_product_kernel_8192_cubed.md.
+KERNEL_DRAM_BYTES_PER_LAUNCH = 2914859776 + 255439360
 
 
 def measured_peaks():
@@ -78,9 +79,10 @@ class ClockSampler:
         for line in self.proc.stdout:
             parts = [p.strip() for p in line.split(",")]
             if len(parts) >= 6:
-                self.samples.append(parts)
+                self.samples.append((time.perf_counter(), parts))
 
-    def stop(self):
+    def stop(self, t_begin=None, t_end=None):
+        """Summary of the samples taken in [t_begin, t_end] (all samples if that window is empty)."""
         if self.proc is None:
             return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
         self.proc.terminate()
@@ -90,7 +92,13 @@ class ClockSampler:
             self.proc.kill()
         sm, mx, reasons = [], [], set()
         names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
-        for s in self.samples:
+        inside = [v for (t, v) in self.samples
+                  if t_begin is not None and t_begin <= t <= t_end + 0.05]
+        window = "timed region"
+        if not inside:
+            inside = [v for (_, v) in self.samples]
+            window = "warm-up and timed region"
+        for s in inside:
             try:
                 sm.append(float(s[0]))
                 mx.append(float(s[1]))
@@ -101,7 +109,24 @@ class ClockSampler:
                     reasons.add(name)
         return {"sm_mhz": statistics.median(sm) if sm else None,
                 "sm_max_mhz": max(mx) if mx else None, "reasons": sorted(reasons),
-                "samples": len(sm)}
+                "samples": len(sm), "window": window}
+
+
+def max_over_ranks(x, world, device):
+    """Max of a per-rank scalar over all ranks (the job is as slow as its slowest rank)."""
+    if world <= 1:
+        return float(x)
+    import torch
+    import torch.distributed as dist
+    t = torch.tensor([float(x)], device=device, dtype=torch.float64)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+def job_throughput(flops_per_rank_step, ms_per_step, world):
+    """Whole-job FP32-equivalent TFLOP/s: every rank runs one full problem per step (independent
+    replicas, weak scaling), and the step time is the max over ranks."""
+    return world * flops_per_rank_step / (ms_per_step * 1e-3) / 1e12
 
 
 def cpu_oracle_sample(rows):
@@ -149,7 +174,7 @@ def run_reference(args, rank):
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--steps", type=int, default=100)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--e2e-steps", type=int, default=3)
@@ -221,21 +246,28 @@ def main():
         def step():
             h.sgemm_cube(A, B, C, SCALE_EXP, binding.TERMWISE)
 
+    sampler = ClockSampler(local_rank)
+    sampler.start()
+    t_warm = time.perf_counter()
     for _ in range(warmup):
         step()
     barrier()
-    sampler = ClockSampler(local_rank)
-    sampler.start()
+    # keep the device busy until nvidia-smi delivers (its first sample takes a few 100 ms), so that
+    # the timed region starts from a loaded, sampled state
+    while not sampler.samples and time.perf_counter() - t_warm < 2.0:
+        step()
+        torch.cuda.synchronize()
     launches0 = h.sgemm_cube_launch_count()
     ev = [torch.cuda.Event(enable_timing=True) for _ in range(args.steps + 1)]
     barrier()
+    t_begin = time.perf_counter()
     ev[0].record()
     for i in range(args.steps):
         step()
         ev[i + 1].record()
     barrier()
     total_ms = ev[0].elapsed_time(ev[-1])
-    clocks = sampler.stop()
+    clocks = sampler.stop(t_begin, time.perf_counter())
     launches = h.sgemm_cube_launch_count() - launches0
     st, det = h.sgemm_cube_check()
     if st != 0:
@@ -250,13 +282,10 @@ def main():
             kernel_samples.append(h.sgemm_cube_last_kernel_ms())
     else:
         kernel_samples = [ev[i].elapsed_time(ev[i + 1]) for i in range(args.steps)]
-    t = torch.tensor([total_ms], device=dev, dtype=torch.float64)
-    if world > 1:
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-    total_ms = float(t.item())
+    total_ms = max_over_ranks(total_ms, world, dev)
     ms_per_step = total_ms / args.steps
     flops = 2.0 * M * N * K
-    value = world * flops / (ms_per_step * 1e-3) / 1e12
+    value = job_throughput(flops, ms_per_step, world)
 
     # Ablation legs on rank 0 (not part of `value`): pre-split kernel, unfused path, split alone.
     extra = {}
@@ -309,10 +338,8 @@ def main():
     for _ in range(args.e2e_steps):
         h.sgemm_cube_host(A_pin, B_pin, C_pin, SCALE_EXP, binding.TERMWISE)
     barrier()
-    e2e_s = torch.tensor([(time.perf_counter() - t0) / args.e2e_steps], device=dev, dtype=torch.float64)
-    if world > 1:
-        dist.all_reduce(e2e_s, op=dist.ReduceOp.MAX)
-    e2e_val = world * flops / float(e2e_s.item()) / 1e12
+    e2e_ms = max_over_ranks((time.perf_counter() - t0) / args.e2e_steps * 1e3, world, dev)
+    e2e_val = job_throughput(flops, e2e_ms, world)
     loss_probe = float(C_pin[0, 0])          # the step's result is read on the host
 
     if rank == 0:
@@ -339,7 +366,7 @@ def main():
                     "d2h_bytes_per_step": 4 * M * N, "result_probe": loss_probe},
             "gpu_launches": int(launches),
             "roofline": {"bound": "tensor", "achieved": achieved, "peak": peak, "unit": "TFLOP/s",
-                         "frac": achieved / peak, "traffic": FUSED_KERNEL_DRAM_BYTES_PER_LAUNCH,
+                         "frac": achieved / peak, "traffic": KERNEL_DRAM_BYTES_PER_LAUNCH if (M == 8192 and args.strategy != "fused") else None,
                          "peak_source": "%s cuBLAS bf16 burst (fp16 has the same nominal rate)"
                                         % peaks["source"],
                          "kernel_ms": kernel_ms,

@@ -67,8 +67,10 @@ enum {
   SGEMM_CUBE_OPT_ELEMENTWISE_K_BLOCK = 1,
   /* 1: run the tensor-core kernels as clusters of two CTAs that share one
    * tcgen05.mma.cta_group::2 (256 x 256 tile per pair, each CTA loading half of the B tile);
-   * 0: one CTA per 128 x 256 tile; 2 (default): pairs when the problem has at least four waves of
-   * pair tiles.  Same arithmetic, bit-identical results either way. */
+   * 0 (default): one CTA per 128 x 256 tile; 2: pairs when the problem has at least four waves
+   * of pair tiles.  Same arithmetic, bit-identical results either way.  (Pairs halve the B-tile
+   * traffic and are the faster mode for k-blocks of 512 and more; at the default k-block of 256
+   * the more frequent TMEM drains cost them more than they save.) */
   SGEMM_CUBE_OPT_CTA_PAIR = 2,
   /* How sgemm_cube computes (same arithmetic and bracketing, bit-identical results):
    * SGEMM_CUBE_STRATEGY_FUSED     one kernel; converter warps split FP32 tiles on the fly, no FP16

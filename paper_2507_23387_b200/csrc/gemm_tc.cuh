@@ -102,10 +102,14 @@ struct TcCfg {
       STAGES * STAGE_BYTES + 1024 /*align*/ + 256 /*barriers*/ + STORE_STAGING;
 };
 
-// Tile rasterisation: groups of 8 tile-rows are walked column by column so that the CTAs
-// running at the same time share A and B tiles in L2.
-__device__ __forceinline__ void tile_coords(int tile, int num_m, int num_n, int& tm, int& tn) {
-  constexpr int kGroupM = 8;
+// Tile rasterisation: groups of `group_m` tile-rows are walked column by column so that the CTAs
+// running at the same time share A and B tiles in L2.  A wave of 148 tiles then covers about
+// group_m x 148 / group_m tiles; its DRAM traffic is the A rows plus the B columns it spans, least
+// when 128 rows x group_m is close to 256 columns x 148 / group_m (16 for 128-row tiles, 8 for
+// the 256-row tiles of CTA pairs).
+__device__ __forceinline__ void tile_coords(int tile, int num_m, int num_n, int& tm, int& tn,
+                                            int group_m = 16) {
+  const int kGroupM = group_m;
   const int per_group = kGroupM * num_n;
   const int group = tile / per_group;
   const int first_m = group * kGroupM;
@@ -229,6 +233,7 @@ __device__ __forceinline__ ConvItem load_item_guarded(const float* __restrict__ 
 
 __device__ __forceinline__ void tmem_ld_cols(uint32_t taddr, uint32_t (&r)[16]) { tmem_ld_32x32b_x16(taddr, r); }
 __device__ __forceinline__ void tmem_ld_cols(uint32_t taddr, uint32_t (&r)[32]) { tmem_ld_32x32b_x32(taddr, r); }
+__device__ __forceinline__ void tmem_ld_cols(uint32_t taddr, uint32_t (&r)[64]) { tmem_ld_32x32b_x64(taddr, r); }
 
 template <int NTERMS, bool FUSED, bool PAIR>
 __global__ void __launch_bounds__(FUSED ? kFusedThreads : kTcThreads, 1)
@@ -309,7 +314,7 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA0, const __grid_constant__
   const int first_tile = PAIR ? (int)(blockIdx.x >> 1) : (int)blockIdx.x;
   const int tile_stride = PAIR ? (int)(gridDim.x >> 1) : (int)gridDim.x;
   auto tile_rc = [&](int tile, int& tm, int& tn) {     // tm in units of 128 rows, tn of 256 columns
-    tile_coords(tile, num_m, num_n, tm, tn);
+    tile_coords(tile, num_m, num_n, tm, tn, PAIR ? 8 : 16);
     if (PAIR) tm = tm * 2 + (int)cta_rank;
   };
   const int num_kb = (p.K + BK - 1) / BK;                      // pipeline stages per tile
@@ -332,9 +337,9 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA0, const __grid_constant__
     uint32_t gchunk = 0;
     bool ok = true;
     float S[128];
-    // TMEM is read 32 columns at a time (fewer, longer loads: the load latency is what a drain
-    // costs), 16 where the register budget is tight.
-    constexpr int GW = FUSED ? 16 : 32;
+    // TMEM is read 64 columns at a time (fewer, longer loads: the tensor pipe is held up for as
+    // long as a drain lasts, and the load latency is most of that), 16 where registers are tight.
+    constexpr int GW = FUSED ? 16 : 64;
     auto wait_tfull = [&](int r) -> bool {
       return mbar_wait_bounded(&tfull_bar[r], drains[r] & 1, abort_flag, p.err, kErrEpiTmemFullWait);
     };

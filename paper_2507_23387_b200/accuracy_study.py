@@ -1,0 +1,158 @@
+"""Accuracy study of SGEMM-cube on the GPU, after the paper's Sec. 6.2 experiments.
+
+Two sweeps, both with the paper's metric (Frobenius-norm relative error against an FP64 product,
+Eq. err, mean over seeds):
+
+  exponent sweep   entries U[-2^e, 2^e] (symmetric) or U[0, 2^e] (non-negative) for a range of
+                   offset exponents e, scale exponents s_b in {0, 6, 11, 12}; compared methods:
+                   termwise and elementwise SGEMM-cube, the hi*hi product alone ("FP16 HGEMM"),
+                   and an FP32 GEMM                                  (Fig. scaling_bit_error)
+  size sweep       error against m = n, against k, and against all three, at offset exponent 0
+                                                                      (Fig. mkn_error)
+
+Everything runs through the library's C ABI (`sgemm_cube`, `sgemm_cube_split`,
+`sgemm_cube_hgemm`); the FP64 reference and the FP32 baseline are torch matmuls on the device.
+Run as a script for a markdown report:
+
+    python -m paper_2507_23387_b200.accuracy_study [--size 1024] [--seeds 5] [--quick]
+"""
+import argparse
+import json
+
+import torch
+
+from . import binding, inputs
+
+
+def frobenius_rel_err(C, C64):
+    d = C.double() - C64
+    return float(d.norm() / C64.norm())
+
+
+def _reference(A, B):
+    return A.double() @ B.double()
+
+
+def _fp32_gemm(A, B):
+    prev = torch.backends.cuda.matmul.allow_tf32
+    torch.backends.cuda.matmul.allow_tf32 = False
+    try:
+        return A @ B
+    finally:
+        torch.backends.cuda.matmul.allow_tf32 = prev
+
+
+def _hgemm_hi_only(h, A, B, s):
+    """hi_A * hi_B alone: what a native FP16 GEMM with FP32 accumulation computes."""
+    M, K = A.shape
+    _, N = B.shape
+    f16 = dict(dtype=torch.float16, device=A.device)
+    Ahi, Alo = torch.empty((M, K), **f16), torch.empty((M, K), **f16)
+    Bhi, Blo = torch.empty((K, N), **f16), torch.empty((K, N), **f16)
+    h.sgemm_cube_split(A, Ahi, Alo, s)
+    h.sgemm_cube_split(B, Bhi, Blo, s)
+    D = torch.empty((M, N), device=A.device)
+    h.sgemm_cube_hgemm(Ahi, Bhi, D)
+    return D
+
+
+def measure(h, A, B, scale_exps=(0, 6, 11, 12)):
+    """Errors of every method on one (A, B) pair; keys like 'termwise_s12'."""
+    C64 = _reference(A, B)
+    M, N = A.shape[0], B.shape[1]
+    out = {"fp32_gemm": frobenius_rel_err(_fp32_gemm(A, B), C64),
+           "fp16_hgemm": frobenius_rel_err(_hgemm_hi_only(h, A, B, 0), C64)}
+    C = torch.empty((M, N), device=A.device)
+    for s in scale_exps:
+        for name, order in (("termwise", binding.TERMWISE), ("elementwise", binding.ELEMENTWISE)):
+            h.sgemm_cube(A, B, C, s, order)
+            out["%s_s%d" % (name, s)] = frobenius_rel_err(C, C64)
+    status, detail = h.sgemm_cube_check()
+    if status != 0:
+        raise RuntimeError("device error %s" % hex(detail))
+    return out
+
+
+def _mean_over_seeds(h, make, seeds, scale_exps):
+    acc = {}
+    for seed in range(seeds):
+        A, B = make(seed)
+        for k, v in measure(h, A, B, scale_exps).items():
+            acc[k] = acc.get(k, 0.0) + v / seeds
+    return acc
+
+
+def exponent_sweep(h, size=1024, exponents=range(-14, 3, 2), seeds=5, nonneg=False,
+                   scale_exps=(0, 6, 11, 12), device="cuda:0"):
+    """Error against the offset exponent e of the inputs (Fig. scaling_bit_error (a) / (b))."""
+    rows = []
+    for e in exponents:
+        def make(seed, e=e):
+            A = torch.from_numpy(inputs.uniform_range(seed, (size, size), e, nonneg, stream=0)).to(device)
+            B = torch.from_numpy(inputs.uniform_range(seed, (size, size), e, nonneg, stream=1)).to(device)
+            return A, B
+        r = _mean_over_seeds(h, make, seeds, scale_exps)
+        r["offset_exponent"] = e
+        rows.append(r)
+    return rows
+
+
+def size_sweep(h, shapes, seeds=5, scale_exp=12, device="cuda:0"):
+    """Error against the matrix sizes at offset exponent 0 (Fig. mkn_error)."""
+    rows = []
+    for (M, N, K) in shapes:
+        def make(seed, M=M, N=N, K=K):
+            A = torch.from_numpy(inputs.uniform_range(seed, (M, K), 0, False, stream=0)).to(device)
+            B = torch.from_numpy(inputs.uniform_range(seed, (K, N), 0, False, stream=1)).to(device)
+            return A, B
+        r = _mean_over_seeds(h, make, seeds, (scale_exp,))
+        r["shape"] = (M, N, K)
+        rows.append(r)
+    return rows
+
+
+def _table(rows, key, cols):
+    lines = ["| %s | %s |" % (key, " | ".join(cols)), "|" + "---|" * (len(cols) + 1)]
+    for r in rows:
+        lines.append("| %s | %s |" % (r[key], " | ".join("%.2e" % r[c] for c in cols)))
+    return "\n".join(lines)
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--size", type=int, default=1024)
+    ap.add_argument("--seeds", type=int, default=5)
+    ap.add_argument("--quick", action="store_true")
+    ap.add_argument("--json", action="store_true")
+    args = ap.parse_args()
+    h = binding.Handle(0)
+    exps = range(-12, 3, 4) if args.quick else range(-16, 5, 2)
+    cols = ["fp16_hgemm", "fp32_gemm", "termwise_s0", "elementwise_s0", "termwise_s6", "termwise_s11",
+            "termwise_s12", "elementwise_s12"]
+    sym = exponent_sweep(h, args.size, exps, args.seeds, nonneg=False)
+    pos = exponent_sweep(h, args.size, exps, args.seeds, nonneg=True)
+    k_fixed = 64 * 44
+    mn = [(n, n, k_fixed) for n in ((512, 2048) if args.quick else (256, 1024, 4096))]
+    ks = [(1024, 1024, k) for k in ((256, 4096) if args.quick else (256, 1024, 4096, 16384, 65536))]
+    alls = [(n, n, n) for n in ((512, 2048) if args.quick else (512, 1024, 2048, 4096))]
+    scol = ["fp16_hgemm", "fp32_gemm", "termwise_s12", "elementwise_s12"]
+    res = {"symmetric": sym, "nonnegative": pos, "vs_mn": size_sweep(h, mn, args.seeds),
+           "vs_k": size_sweep(h, ks, args.seeds), "vs_all": size_sweep(h, alls, args.seeds)}
+    h.destroy()
+    if args.json:
+        print(json.dumps(res))
+        return
+    print("## Relative error vs offset exponent, U[-2^e, 2^e], %d^3, %d seeds\n" % (args.size, args.seeds))
+    print(_table(sym, "offset_exponent", cols))
+    print("\n## Relative error vs offset exponent, U[0, 2^e]\n")
+    print(_table(pos, "offset_exponent", cols))
+    print("\n## Relative error vs m = n (k = %d), offset exponent 0, s_b = 12\n" % k_fixed)
+    print(_table(res["vs_mn"], "shape", scol))
+    print("\n## Relative error vs k (m = n = 1024)\n")
+    print(_table(res["vs_k"], "shape", scol))
+    print("\n## Relative error vs m = n = k\n")
+    print(_table(res["vs_all"], "shape", scol))
+
+
+if __name__ == "__main__":
+    main()

@@ -47,7 +47,7 @@ struct sgemm_cube_ctx {
   void* host_ws = nullptr;     // host-buffer path: device copies of A, B, C
   size_t host_ws_bytes = 0;
   long long launches = 0;
-  int kblock_termwise = 256;
+  int kblock_termwise = 128;
   int kblock_elementwise = 64;
   int cta_pair = 0;            // 0/1: never/always 2-CTA clusters (cta_group::2); 2: by problem size
   int strategy = 0;            // sgemm_cube: 0 auto, 1 fused kernel, 2 split kernel + 3-product kernel
@@ -275,7 +275,7 @@ int launch_two_phase(sgemm_cube_ctx* h, int M, int N, int K, const float* A, int
 int launch_sgemm_cube(sgemm_cube_ctx* h, int M, int N, int K, const float* A, int64_t lda, const float* B,
                       int64_t ldb, float* C, int64_t ldc, int s, int order, cudaStream_t st) {
   bool two_phase = (h->strategy == 2) ||
-                   (h->strategy == 0 && (double)M * (double)N * (double)K >= 1024.0 * 1024.0 * 1024.0);
+                   (h->strategy == 0 && (double)M * (double)N * (double)K >= 512.0 * 512.0 * 512.0);
   if (two_phase) {
     int rc = launch_two_phase(h, M, N, K, A, lda, B, ldb, C, ldc, s, order, st);
     if (rc != SGEMM_CUBE_ALLOC_FAILED || h->strategy == 2) return rc;

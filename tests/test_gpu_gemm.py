@@ -102,6 +102,17 @@ def test_config1_256_cubed_uniform(handle, path, order, seed):
 
 
 @pytest.mark.parametrize("path,order", PATHS)
+@pytest.mark.parametrize("K", [1024, 4096])
+def test_one_signed_inputs(handle, path, order, K):
+    # U[0, 1) entries (the paper's non-negative sampling): no cancellation, so the truncation of
+    # the tensor core's accumulator shows as a bias.  Same gates as everywhere else.
+    A = inputs.uniform_range(2, (256, K), 0, True, stream=0)
+    B = inputs.uniform_range(2, (K, 512), 0, True, stream=1)
+    C = run(handle, path, to_dev(A), to_dev(B), 11, order)
+    gates(C, A, B, 11, order, label="nonneg %s K=%d" % (path, K))
+
+
+@pytest.mark.parametrize("path,order", PATHS)
 @pytest.mark.parametrize("shape", [(1, 1, 1), (129, 257, 33), (200, 300, 136), (384, 768, 1000),
                                    (127, 8, 2049), (640, 1280, 96)])
 def test_ragged_shapes(handle, path, order, shape):

@@ -193,6 +193,32 @@ int sgemm_cube_host(sgemm_cube_handle h, int M, int N, int K,
                     float* C_host, int64_t ldc,
                     int scale_exp, int accumulation_order, void* stream);
 
+/* Exponent window of a matrix's FP16 high words (paper Sec. 4.2: e_min and e_max of
+ * Eq. sf_bounds are the smallest and largest unbiased exponents E' - 15 of the finite high
+ * components).  One pass over X on the device; the call synchronises `stream` and writes to HOST
+ * memory:
+ *   window_out[0] = e_min, window_out[1] = e_max over the NORMAL high words (127 / -127 if none),
+ *   window_out[2] = number of entries whose high word is subnormal (|x| < 2^-14: the 22-bit
+ *                   guarantee cannot be kept by scaling the residual alone, Sec. 4.2),
+ *   window_out[3] = number of entries whose high word is inf or NaN (|x| >= 65520),
+ *   window_out[4] = number of entries whose high word is zero.
+ *   X_dev rows x cols FP32, ldx >= cols (device, read); window_out 5 x int64 (host, written).
+ * Errors: INVALID_ARG, CUDA_ERROR. */
+int sgemm_cube_exponent_window(sgemm_cube_handle h, int rows, int cols,
+                               const float* X_dev, int64_t ldx,
+                               int64_t* window_out, void* stream);
+
+/* Scale exponent for a pair of operands from their exponent windows (host arithmetic only).
+ * Eq. sf_bounds:  -3 - e_min <= s_b <= 26 - e_max  over both operands; following Sec. 4.2 ("scale
+ * the residual as far from the underflow threshold as the largest entry permits") the upper end
+ * is taken, capped at 15:  *scale_exp_out = min(26 - e_max, 15).  Full normal FP16 range
+ * (e_max = 15) gives 11, e_max <= 14 gives at least 12.
+ * *protected_out (optional) = 1 if that value also satisfies the lower end and no high word is
+ * subnormal, inf or NaN, i.e. if Eq. split_error holds for every entry; else 0.
+ * Errors: INVALID_ARG. */
+int sgemm_cube_choose_scale_exp(const int64_t* window_a, const int64_t* window_b,
+                                int* scale_exp_out, int* protected_out);
+
 /* Size in bytes of the fixed device scratch area used by sgemm_cube_unfused_static. */
 #define SGEMM_CUBE_STATIC_SCRATCH_BYTES (32u << 20)
 

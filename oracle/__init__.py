@@ -163,3 +163,20 @@ def componentwise_err(C, C64, ABabs):
     if np.all(zero):
         return 0.0
     return float((d[~zero] / ABabs[~zero]).max())
+
+
+def exponent_window(X):
+    """[e_min, e_max, #subnormal hi, #non-finite hi, #zero hi] of the FP16 high words of X:
+    the exponents E' - 15 that Eq. sf_bounds is stated on (Sec. 4.2)."""
+    hi, _ = split(np.atleast_2d(np.asarray(X, dtype=np.float32)), 0)
+    E = (hi.astype(np.int64) >> 10) & 0x1F
+    Mant = hi.astype(np.int64) & 0x3FF
+    normal = (E > 0) & (E < 0x1F)
+    e = E[normal] - 15
+    return [int(e.min()) if e.size else 127, int(e.max()) if e.size else -127,
+            int(((E == 0) & (Mant != 0)).sum()), int((E == 0x1F).sum()), int(((E == 0) & (Mant == 0)).sum())]
+
+
+def scale_exp_bounds(e_min, e_max):
+    """Eq. sf_bounds: -3 - e_min <= s_b <= 26 - e_max."""
+    return -3 - e_min, 26 - e_max

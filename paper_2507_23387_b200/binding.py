@@ -21,6 +21,7 @@ STRATEGY_AUTO, STRATEGY_FUSED, STRATEGY_TWO_PHASE = 0, 1, 2
 EXPORTS = ["sgemm_cube_create", "sgemm_cube_destroy", "sgemm_cube_set_option", "sgemm_cube_split",
            "sgemm_cube", "sgemm_cube_unfused", "sgemm_cube_presplit", "sgemm_cube_hgemm",
            "sgemm_cube_host", "sgemm_cube_unfused_static", "sgemm_cube_check", "sgemm_cube_launch_count", "sgemm_cube_last_kernel_ms",
+           "sgemm_cube_exponent_window", "sgemm_cube_choose_scale_exp",
            "sgemm_cube_status_string", "sgemm_cube_version"]
 
 _lib = None
@@ -56,6 +57,9 @@ def load():
     lib.sgemm_cube_unfused_static.argtypes = [i32, i32, i32, vp, i64, vp, i64, vp, i64, i32, vp]
     lib.sgemm_cube_check.argtypes = [vp, vp, ctypes.POINTER(ctypes.c_uint32)]
     lib.sgemm_cube_last_kernel_ms.argtypes = [vp, ctypes.POINTER(ctypes.c_float)]
+    lib.sgemm_cube_exponent_window.argtypes = [vp, i32, i32, vp, i64, ctypes.POINTER(i64), vp]
+    lib.sgemm_cube_choose_scale_exp.argtypes = [ctypes.POINTER(i64), ctypes.POINTER(i64),
+                                                ctypes.POINTER(i32), ctypes.POINTER(i32)]
     lib.sgemm_cube_launch_count.argtypes = [vp]
     lib.sgemm_cube_launch_count.restype = i64
     lib.sgemm_cube_status_string.argtypes = [i32]
@@ -109,6 +113,16 @@ def sgemm_cube_unfused_static(A, B, C, scale_exp=11, stream=None):
                                             _dev(B, torch.float32), _ld(B), _dev(C, torch.float32),
                                             _ld(C), scale_exp, _stream_ptr(stream)),
            "sgemm_cube_unfused_static")
+
+
+def sgemm_cube_choose_scale_exp(window_a, window_b):
+    """(scale_exp, protected) for two exponent windows (see Handle.sgemm_cube_exponent_window)."""
+    wa = (ctypes.c_int64 * 5)(*[int(v) for v in window_a])
+    wb = (ctypes.c_int64 * 5)(*[int(v) for v in window_b])
+    s, prot = ctypes.c_int(0), ctypes.c_int(0)
+    _check(load().sgemm_cube_choose_scale_exp(wa, wb, ctypes.byref(s), ctypes.byref(prot)),
+           "sgemm_cube_choose_scale_exp")
+    return int(s.value), bool(prot.value)
 
 
 class Handle:
@@ -189,6 +203,14 @@ class Handle:
         detail = ctypes.c_uint32(0)
         st = load().sgemm_cube_check(self._h, _stream_ptr(stream), ctypes.byref(detail))
         return int(st), int(detail.value)
+
+    def sgemm_cube_exponent_window(self, X, stream=None):
+        """[e_min, e_max, #subnormal hi, #non-finite hi, #zero hi] of a device matrix."""
+        rows, cols = X.shape
+        out = (ctypes.c_int64 * 5)()
+        _check(load().sgemm_cube_exponent_window(self._h, rows, cols, _dev(X, torch.float32), _ld(X),
+                                                 out, _stream_ptr(stream)), "sgemm_cube_exponent_window")
+        return [int(v) for v in out]
 
     def sgemm_cube_launch_count(self) -> int:
         return int(load().sgemm_cube_launch_count(self._h))

@@ -41,7 +41,7 @@ inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 
 struct sgemm_cube_ctx {
   int device = 0;
   int sm_count = 0;
-  unsigned int* err_dev = nullptr;
+  unsigned int* err_dev = nullptr;   // [0] error word; [4..8] scratch of sgemm_cube_exponent_window
   void* ws = nullptr;          // unfused path: FP16 words of A and B, D_hh, D_x
   size_t ws_bytes = 0;
   void* host_ws = nullptr;     // host-buffer path: device copies of A, B, C
@@ -331,12 +331,12 @@ int sgemm_cube_create(sgemm_cube_handle* out, int device) {
     return SGEMM_CUBE_CUDA_ERROR;
   }
   h->encode = reinterpret_cast<EncodeTiledFn>(fn);
-  if (cudaMalloc(reinterpret_cast<void**>(&h->err_dev), sizeof(unsigned int)) != cudaSuccess) {
+  if (cudaMalloc(reinterpret_cast<void**>(&h->err_dev), 16 * sizeof(unsigned int)) != cudaSuccess) {
     cudaGetLastError();
     delete h;
     return SGEMM_CUBE_ALLOC_FAILED;
   }
-  if (cudaMemset(h->err_dev, 0, sizeof(unsigned int)) != cudaSuccess) {
+  if (cudaMemset(h->err_dev, 0, 16 * sizeof(unsigned int)) != cudaSuccess) {
     cudaFree(h->err_dev);
     delete h;
     return SGEMM_CUBE_CUDA_ERROR;
@@ -540,6 +540,61 @@ int sgemm_cube_check(sgemm_cube_handle h, void* stream, uint32_t* detail_out) {
   if (e) {
     cudaMemset(h->err_dev, 0, sizeof(e));
     return SGEMM_CUBE_DEVICE_TIMEOUT;
+  }
+  return SGEMM_CUBE_OK;
+}
+
+int sgemm_cube_exponent_window(sgemm_cube_handle h, int rows, int cols, const float* X, int64_t ldx,
+                               int64_t* window_out, void* stream) {
+  if (!h || !X || !window_out) return SGEMM_CUBE_INVALID_ARG;
+  if (rows <= 0 || cols <= 0 || ldx < cols) return SGEMM_CUBE_INVALID_ARG;
+  DeviceGuard g(h->device);
+  if (!g.ok) return SGEMM_CUBE_CUDA_ERROR;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  long long* dev = reinterpret_cast<long long*>(h->err_dev + 4);
+  const long long init[5] = {127, -127, 0, 0, 0};
+  if (cudaMemcpyAsync(dev, init, sizeof(init), cudaMemcpyHostToDevice, st) != cudaSuccess) {
+    cudaGetLastError();
+    return SGEMM_CUBE_CUDA_ERROR;
+  }
+  const long long total = (long long)rows * cols;
+  long long blocks = (total + 1023) / 1024;
+  const long long cap = (long long)h->sm_count * 16;
+  if (blocks > cap) blocks = cap;
+  sgc::exponent_window_kernel<<<(unsigned)blocks, 256, 0, st>>>(rows, cols, X, ldx, dev);
+  h->launches++;
+  if (cudaGetLastError() != cudaSuccess) return SGEMM_CUBE_CUDA_ERROR;
+  long long res[5];
+  if (cudaMemcpyAsync(res, dev, sizeof(res), cudaMemcpyDeviceToHost, st) != cudaSuccess ||
+      cudaStreamSynchronize(st) != cudaSuccess) {
+    cudaGetLastError();
+    return SGEMM_CUBE_CUDA_ERROR;
+  }
+  for (int i = 0; i < 5; ++i) window_out[i] = res[i];
+  return SGEMM_CUBE_OK;
+}
+
+int sgemm_cube_choose_scale_exp(const int64_t* window_a, const int64_t* window_b, int* scale_exp_out,
+                                int* protected_out) {
+  if (!window_a || !window_b || !scale_exp_out) return SGEMM_CUBE_INVALID_ARG;
+  const bool any_a = window_a[1] >= window_a[0], any_b = window_b[1] >= window_b[0];
+  int e_max = -127, e_min = 127;
+  if (any_a) { e_max = (int)window_a[1]; e_min = (int)window_a[0]; }
+  if (any_b) {
+    e_max = (int)window_b[1] > e_max ? (int)window_b[1] : e_max;
+    e_min = (int)window_b[0] < e_min ? (int)window_b[0] : e_min;
+  }
+  int s = 15;                                  // nothing normal and finite: any scale will do
+  if (any_a || any_b) {
+    s = 26 - e_max;                            // Rule 2 / upper end of Eq. sf_bounds
+    if (s > 15) s = 15;
+    if (s < 0) s = 0;
+  }
+  *scale_exp_out = s;
+  if (protected_out) {
+    const bool clean = window_a[2] == 0 && window_a[3] == 0 && window_b[2] == 0 && window_b[3] == 0;
+    const bool lower_ok = !(any_a || any_b) || s >= -3 - e_min;    // lower end of Eq. sf_bounds
+    *protected_out = (clean && lower_ok) ? 1 : 0;
   }
   return SGEMM_CUBE_OK;
 }

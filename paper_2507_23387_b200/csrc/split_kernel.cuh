@@ -92,4 +92,44 @@ combine_kernel(int rows, int cols, const float* __restrict__ Dhh, const float* _
   }
 }
 
+// Exponent window of the FP16 high words of a matrix (Sec. 4.2: e_min and e_max of Eq. sf_bounds
+// are the smallest and largest unbiased exponents E' - 15 of the finite, normal high components).
+// out[0] = min exponent, out[1] = max exponent over normal high words (initialised by the caller to
+// +127 / -127), out[2] = number of entries whose high word is subnormal (non-zero), out[3] =
+// number of entries whose high word is inf or NaN, out[4] = number of zero high words.
+// HBM-bound: 4 bytes read per element.
+__global__ void __launch_bounds__(256)
+exponent_window_kernel(int rows, int cols, const float* __restrict__ X, long long ldx,
+                       long long* out) {
+  int emin = 127, emax = -127;
+  unsigned int n_sub = 0, n_nonfinite = 0, n_zero = 0;      // per thread: < 2^32 elements each
+  const long long total = (long long)rows * cols;
+  const long long stride = (long long)gridDim.x * blockDim.x;
+  for (long long it = (long long)blockIdx.x * blockDim.x + threadIdx.x; it < total; it += stride) {
+    const long long r = it / cols;
+    const long long c = it - r * cols;
+    const unsigned int h = __half_as_ushort(__float2half_rn(__ldg(X + r * ldx + c)));
+    const int E = (h >> 10) & 0x1F;
+    const int M = h & 0x3FF;
+    if (E == 0x1F) ++n_nonfinite;
+    else if (E == 0) { if (M) ++n_sub; else ++n_zero; }
+    else { emin = min(emin, E - 15); emax = max(emax, E - 15); }
+  }
+  for (int o = 16; o > 0; o >>= 1) {
+    emin = min(emin, __shfl_xor_sync(0xffffffffu, emin, o));
+    emax = max(emax, __shfl_xor_sync(0xffffffffu, emax, o));
+    n_sub += __shfl_xor_sync(0xffffffffu, n_sub, o);
+    n_nonfinite += __shfl_xor_sync(0xffffffffu, n_nonfinite, o);
+    n_zero += __shfl_xor_sync(0xffffffffu, n_zero, o);
+  }
+  if ((threadIdx.x & 31) == 0) {
+    atomicMin(&out[0], (long long)emin);
+    atomicMax(&out[1], (long long)emax);
+    unsigned long long* cnt = reinterpret_cast<unsigned long long*>(out);
+    if (n_sub) atomicAdd(&cnt[2], (unsigned long long)n_sub);
+    if (n_nonfinite) atomicAdd(&cnt[3], (unsigned long long)n_nonfinite);
+    if (n_zero) atomicAdd(&cnt[4], (unsigned long long)n_zero);
+  }
+}
+
 }  // namespace sgc

@@ -256,7 +256,8 @@ def test_config4_error_growth_termwise_vs_elementwise(handle):
         assert res[(65536, order)] < 4 * 8 * res[(1024, order)]
 
 
-@pytest.mark.parametrize("shape", [(16384, 16384, 1024), (12288, 12288, 12288)])
+@pytest.mark.parametrize("shape", [(2048, 2048, 2048), (16384, 16384, 1024), (12288, 12288, 12288),
+                                   (16384, 16384, 16384)])
 def test_config5_large_shapes_sampled_rows(handle, shape):
     M, N, K = shape
     A = inputs.device_normal(0, (M, K))

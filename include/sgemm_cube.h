@@ -184,7 +184,11 @@ int sgemm_cube_hgemm(sgemm_cube_handle h, int M, int N, int K,
 /* Host-buffer convenience around sgemm_cube: copies A and B from HOST memory to the handle's
  * device workspace, runs the fused kernel, copies C back to HOST memory and synchronises the
  * stream before returning.  Pinned host memory makes the copies asynchronous to the host but the
- * call still returns only when C_host is complete.
+ * call still returns only when C_host is complete.  For M >= 1024 and M*N*K >= 2^30 (and a
+ * strategy other than FUSED) the call is pipelined: B is copied and split once, A and C move in
+ * about eight row panels on two internal copy streams so that the upload of one panel, the
+ * products of the previous one and the download of the one before overlap.  The result is
+ * bit-identical to sgemm_cube on device copies of the same operands.
  *   A_host M x K (lda >= K), B_host K x N (ldb >= N), C_host M x N (ldc >= N), all FP32 HOST.
  * Errors: INVALID_ARG, ALLOC_FAILED, CUDA_ERROR, DEVICE_TIMEOUT. */
 int sgemm_cube_host(sgemm_cube_handle h, int M, int N, int K,

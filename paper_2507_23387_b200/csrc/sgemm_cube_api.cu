@@ -54,6 +54,11 @@ struct sgemm_cube_ctx {
   int time_kernel = 0;         // record events around the tensor-core kernel of sgemm_cube
   cudaEvent_t ev0 = nullptr, ev1 = nullptr;
   bool ev_recorded = false;
+  // host-buffer path: copy streams and events of the panel pipeline (created on first use)
+  static constexpr int kMaxPanels = 32;
+  cudaStream_t s_in = nullptr, s_out = nullptr;
+  cudaEvent_t ev_start = nullptr, ev_b = nullptr, ev_out = nullptr;
+  cudaEvent_t ev_a[kMaxPanels] = {}, ev_c[kMaxPanels] = {};
   int max_pair_clusters[3] = {0, 0, 0};   // co-resident 2-CTA clusters: <1,false>, <3,false>, <3,true>
   EncodeTiledFn encode = nullptr;
   bool attrs_set = false;
@@ -287,6 +292,10 @@ int launch_sgemm_cube(sgemm_cube_ctx* h, int M, int N, int K, const float* A, in
   return rc;
 }
 
+int host_pipelined(sgemm_cube_ctx* h, int M, int N, int K, const float* A_host, int64_t lda,
+                   const float* B_host, int64_t ldb, float* C_host, int64_t ldc, int s, int order,
+                   cudaStream_t st, float* dA, size_t ldA, float* dB, size_t ldB, float* dC, size_t ldC);
+
 }  // namespace
 
 extern "C" {
@@ -357,6 +366,15 @@ int sgemm_cube_destroy(sgemm_cube_handle h) {
   if (h->host_ws) cudaFree(h->host_ws);
   if (h->ev0) cudaEventDestroy(h->ev0);
   if (h->ev1) cudaEventDestroy(h->ev1);
+  if (h->s_in) cudaStreamDestroy(h->s_in);
+  if (h->s_out) cudaStreamDestroy(h->s_out);
+  if (h->ev_start) cudaEventDestroy(h->ev_start);
+  if (h->ev_b) cudaEventDestroy(h->ev_b);
+  if (h->ev_out) cudaEventDestroy(h->ev_out);
+  for (int i = 0; i < sgemm_cube_ctx::kMaxPanels; ++i) {
+    if (h->ev_a[i]) cudaEventDestroy(h->ev_a[i]);
+    if (h->ev_c[i]) cudaEventDestroy(h->ev_c[i]);
+  }
   cudaFree(h->err_dev);
   delete h;
   return rc;
@@ -511,6 +529,14 @@ int sgemm_cube_host(sgemm_cube_handle h, int M, int N, int K, const float* A_hos
   float* dA = reinterpret_cast<float*>(w);
   float* dB = reinterpret_cast<float*>(w + szA);
   float* dC = reinterpret_cast<float*>(w + szA + szB);
+  if (h->strategy != SGEMM_CUBE_STRATEGY_FUSED && M >= 1024 &&
+      (double)M * (double)N * (double)K >= 1024.0 * 1024.0 * 1024.0) {
+    rc = host_pipelined(h, M, N, K, A_host, lda, B_host, ldb, C_host, ldc, scale_exp, order, st, dA, ldA,
+                        dB, ldB, dC, ldC);
+    if (rc == SGEMM_CUBE_OK) return sgemm_cube_check(h, stream, nullptr);
+    if (rc != SGEMM_CUBE_ALLOC_FAILED) return rc;
+    // no room for the FP16 words: fall through to the plain sequence below
+  }
   if (cudaMemcpy2DAsync(dA, ldA * 4, A_host, (size_t)lda * 4, (size_t)K * 4, M, cudaMemcpyHostToDevice, st) != cudaSuccess ||
       cudaMemcpy2DAsync(dB, ldB * 4, B_host, (size_t)ldb * 4, (size_t)N * 4, K, cudaMemcpyHostToDevice, st) != cudaSuccess) {
     cudaGetLastError();
@@ -524,6 +550,87 @@ int sgemm_cube_host(sgemm_cube_handle h, int M, int N, int K, const float* A_hos
   }
   return sgemm_cube_check(h, stream, nullptr);
 }
+
+}  // extern "C"
+
+namespace {
+
+int host_pipeline_setup(sgemm_cube_ctx* h) {
+  if (h->s_in) return SGEMM_CUBE_OK;
+  bool ok = cudaStreamCreateWithFlags(&h->s_in, cudaStreamNonBlocking) == cudaSuccess &&
+            cudaStreamCreateWithFlags(&h->s_out, cudaStreamNonBlocking) == cudaSuccess &&
+            cudaEventCreateWithFlags(&h->ev_start, cudaEventDisableTiming) == cudaSuccess &&
+            cudaEventCreateWithFlags(&h->ev_b, cudaEventDisableTiming) == cudaSuccess &&
+            cudaEventCreateWithFlags(&h->ev_out, cudaEventDisableTiming) == cudaSuccess;
+  for (int i = 0; ok && i < sgemm_cube_ctx::kMaxPanels; ++i)
+    ok = cudaEventCreateWithFlags(&h->ev_a[i], cudaEventDisableTiming) == cudaSuccess &&
+         cudaEventCreateWithFlags(&h->ev_c[i], cudaEventDisableTiming) == cudaSuccess;
+  if (!ok) { cudaGetLastError(); return SGEMM_CUBE_CUDA_ERROR; }
+  return SGEMM_CUBE_OK;
+}
+
+// Host-buffer path for large problems: B is copied and split once; A and C move in row panels so
+// that the upload of panel p + 1, the products of panel p and the download of panel p - 1 overlap
+// (one copy stream per direction besides the caller's stream).  Same kernels, same per-element
+// arithmetic as sgemm_cube's two-phase strategy: a row panel of C depends on its rows of A only.
+int host_pipelined(sgemm_cube_ctx* h, int M, int N, int K, const float* A_host, int64_t lda,
+                   const float* B_host, int64_t ldb, float* C_host, int64_t ldc, int s, int order,
+                   cudaStream_t st, float* dA, size_t ldA, float* dB, size_t ldB, float* dC, size_t ldC) {
+  int rc = host_pipeline_setup(h);
+  if (rc) return rc;
+  const size_t ldA16 = round_up((size_t)K, 8), ldB16 = round_up((size_t)N, 8);
+  const size_t szA = round_up((size_t)M * ldA16 * 2, 256), szB = round_up((size_t)K * ldB16 * 2, 256);
+  rc = grow(&h->ws, &h->ws_bytes, 2 * szA + 2 * szB);
+  if (rc) return rc;
+  uint8_t* w = static_cast<uint8_t*>(h->ws);
+  uint16_t* Ahi = reinterpret_cast<uint16_t*>(w);
+  uint16_t* Alo = reinterpret_cast<uint16_t*>(w + szA);
+  uint16_t* Bhi = reinterpret_cast<uint16_t*>(w + 2 * szA);
+  uint16_t* Blo = reinterpret_cast<uint16_t*>(w + 2 * szA + szB);
+  int panel = (int)round_up((size_t)(M + 7) / 8, 256);           // about eight panels
+  while ((M + panel - 1) / panel > sgemm_cube_ctx::kMaxPanels) panel *= 2;
+  const int panels = (M + panel - 1) / panel;
+  const int kblock = (order == SGEMM_CUBE_TERMWISE) ? h->kblock_termwise : h->kblock_elementwise;
+  const float inv = ldexpf(1.0f, -s);
+  bool ok = true;
+  // the copy streams start after whatever the caller's stream holds (earlier users of the buffers)
+  ok = ok && cudaEventRecord(h->ev_start, st) == cudaSuccess;
+  ok = ok && cudaStreamWaitEvent(h->s_in, h->ev_start, 0) == cudaSuccess;
+  ok = ok && cudaStreamWaitEvent(h->s_out, h->ev_start, 0) == cudaSuccess;
+  ok = ok && cudaMemcpy2DAsync(dB, ldB * 4, B_host, (size_t)ldb * 4, (size_t)N * 4, K,
+                               cudaMemcpyHostToDevice, h->s_in) == cudaSuccess;
+  ok = ok && cudaEventRecord(h->ev_b, h->s_in) == cudaSuccess;
+  ok = ok && cudaStreamWaitEvent(st, h->ev_b, 0) == cudaSuccess;
+  if (!ok) { cudaGetLastError(); return SGEMM_CUBE_CUDA_ERROR; }
+  if ((rc = launch_split(h, K, N, dB, (int64_t)ldB, Bhi, Blo, (int64_t)ldB16, s, st))) return rc;
+  for (int p = 0; p < panels; ++p) {
+    const int r0 = p * panel;
+    const int rows = (M - r0 < panel) ? (M - r0) : panel;
+    ok = ok && cudaMemcpy2DAsync(dA + (size_t)r0 * ldA, ldA * 4, A_host + (size_t)r0 * lda, (size_t)lda * 4,
+                                 (size_t)K * 4, rows, cudaMemcpyHostToDevice, h->s_in) == cudaSuccess;
+    ok = ok && cudaEventRecord(h->ev_a[p], h->s_in) == cudaSuccess;
+    ok = ok && cudaStreamWaitEvent(st, h->ev_a[p], 0) == cudaSuccess;
+    if (!ok) { cudaGetLastError(); return SGEMM_CUBE_CUDA_ERROR; }
+    if ((rc = launch_split(h, rows, K, dA + (size_t)r0 * ldA, (int64_t)ldA, Ahi + (size_t)r0 * ldA16,
+                           Alo + (size_t)r0 * ldA16, (int64_t)ldA16, s, st))) return rc;
+    if ((rc = launch_tc_gemm<3>(h, rows, N, K, Ahi + (size_t)r0 * ldA16, Alo + (size_t)r0 * ldA16,
+                                (int64_t)ldA16, Bhi, Blo, (int64_t)ldB16, dC + (size_t)r0 * ldC, (int64_t)ldC,
+                                0, order, kblock, inv, st))) return rc;
+    ok = ok && cudaEventRecord(h->ev_c[p], st) == cudaSuccess;
+    ok = ok && cudaStreamWaitEvent(h->s_out, h->ev_c[p], 0) == cudaSuccess;
+    ok = ok && cudaMemcpy2DAsync(C_host + (size_t)r0 * ldc, (size_t)ldc * 4, dC + (size_t)r0 * ldC, ldC * 4,
+                                 (size_t)N * 4, rows, cudaMemcpyDeviceToHost, h->s_out) == cudaSuccess;
+    if (!ok) { cudaGetLastError(); return SGEMM_CUBE_CUDA_ERROR; }
+  }
+  ok = ok && cudaEventRecord(h->ev_out, h->s_out) == cudaSuccess;
+  ok = ok && cudaStreamWaitEvent(st, h->ev_out, 0) == cudaSuccess;
+  if (!ok) { cudaGetLastError(); return SGEMM_CUBE_CUDA_ERROR; }
+  return SGEMM_CUBE_OK;
+}
+
+}  // namespace
+
+extern "C" {
 
 int sgemm_cube_check(sgemm_cube_handle h, void* stream, uint32_t* detail_out) {
   if (!h) return SGEMM_CUBE_INVALID_ARG;

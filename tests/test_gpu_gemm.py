@@ -319,11 +319,19 @@ def test_argument_errors(handle):
     assert handle.sgemm_cube_check()[0] == 0
 
 
-def test_host_buffer_entry_point(handle):
-    M, N, K = 300, 520, 200
+@pytest.mark.parametrize("shape", [(300, 520, 200), (1500, 1030, 1000), (2048, 1024, 1024)])
+def test_host_buffer_entry_point(handle, shape):
+    # small: plain copy-compute-copy; the two larger shapes take the panel pipeline (ragged last
+    # panel and ragged tiles in the middle one).  Either way bit-identical to the device call.
+    M, N, K = shape
     A, B = inputs.make_pair("normal", 8, M, N, K)
     Ah, Bh = torch.from_numpy(A).pin_memory(), torch.from_numpy(B).pin_memory()
-    Ch = torch.empty((M, N)).pin_memory()
-    handle.sgemm_cube_host(Ah, Bh, Ch, 11, T)
-    Cd = run(handle, "fused", padded_dev(A, 4), padded_dev(B, 4), 11, T)
-    assert np.array_equal(Ch.numpy(), Cd)
+    Ch = torch.full((M, N), float("nan")).pin_memory()
+    for order in (T, E):
+        handle.sgemm_cube_host(Ah, Bh, Ch, 11, order)
+        Cd = run(handle, "auto", padded_dev(A, 4), padded_dev(B, 4), 11, order)
+        assert np.array_equal(Ch.numpy(), Cd)
+    # pageable host memory works too (the copies are then staged by the driver)
+    C2 = torch.empty((M, N))
+    handle.sgemm_cube_host(torch.from_numpy(A), torch.from_numpy(B), C2, 11, T)
+    assert np.array_equal(C2.numpy(), run(handle, "auto", padded_dev(A, 4), padded_dev(B, 4), 11, T))

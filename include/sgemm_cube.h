@@ -73,11 +73,13 @@ enum {
   /* 1: run the tensor-core kernels as clusters of two CTAs that share one
    * tcgen05.mma.cta_group::2 (256 x 256 tile per pair, each CTA loading half of the B tile);
    * 0 (default): one CTA per 128 x 256 tile; 2: pairs when the problem has at least four waves
-   * of pair tiles.  Same arithmetic, bit-identical results either way.  (Pairs halve the B-tile
+   * of pair tiles.  Same arithmetic, bit-identical results either way as long as split-K (below,
+   * single CTAs only) does not apply.  (Pairs halve the B-tile
    * traffic and are the faster mode for k-blocks of 512 and more; at the default k-block of 256
    * the more frequent TMEM drains cost them more than they save.) */
   SGEMM_CUBE_OPT_CTA_PAIR = 2,
-  /* How sgemm_cube computes (same arithmetic and bracketing, bit-identical results):
+  /* How sgemm_cube computes (same arithmetic; same bracketing and bit-identical results except
+   * where split-K, which only the two-phase strategy uses, re-brackets the k-block sums):
    * SGEMM_CUBE_STRATEGY_FUSED     one kernel; converter warps split FP32 tiles on the fly, no FP16
    *                               copy of A or B exists in device memory, no workspace;
    * SGEMM_CUBE_STRATEGY_TWO_PHASE the split kernel writes the FP16 words of A and B once into the
@@ -89,7 +91,15 @@ enum {
   SGEMM_CUBE_OPT_STRATEGY = 3,
   /* 1: sgemm_cube records CUDA events around its tensor-core kernel, for
    * sgemm_cube_last_kernel_ms.  Default 0. */
-  SGEMM_CUBE_OPT_TIME_KERNEL = 4
+  SGEMM_CUBE_OPT_TIME_KERNEL = 4,
+  /* 1 (default): when a problem has so few 128 x 256 tiles that more than half of the SMs would
+   * idle and k is long enough, the three-product kernel (two-phase sgemm_cube,
+   * sgemm_cube_presplit) cuts the k range into up to 16 slices of whole k-blocks, one work unit per
+   * (tile, slice); the slices' sums go to a workspace (grown with cudaMalloc on first use) and a
+   * reduction kernel adds them in slice order (termwise: hi*hi sums and correction sums
+   * separately, combined once).  This is one more level of the blocked summation of Sec. 4.5 and
+   * is deterministic.  0: never split. */
+  SGEMM_CUBE_OPT_SPLIT_K = 5
 };
 
 enum {
@@ -131,7 +141,7 @@ int sgemm_cube_split(sgemm_cube_handle h, int rows, int cols,
  * cores with FP32 accumulation, the reconstruction in FP32; C overwritten (no alpha/beta).
  * The operand split runs either inside the product kernel (converter warps, no FP16 copy of A or
  * B in device memory) or once up front into the handle's workspace: see SGEMM_CUBE_OPT_STRATEGY.
- * Both give bit-identical C.
+ * Both give bit-identical C unless split-K applies (SGEMM_CUBE_OPT_SPLIT_K).
  *   A_dev  M x K FP32, lda >= K     (device, read)
  *   B_dev  K x N FP32, ldb >= N     (device, read)
  *   C_dev  M x N FP32, ldc >= N     (device, written)
@@ -188,7 +198,9 @@ int sgemm_cube_hgemm(sgemm_cube_handle h, int M, int N, int K,
  * strategy other than FUSED) the call is pipelined: B is copied and split once, A and C move in
  * about eight row panels on two internal copy streams so that the upload of one panel, the
  * products of the previous one and the download of the one before overlap.  The result is
- * bit-identical to sgemm_cube on device copies of the same operands.
+ * bit-identical to sgemm_cube on device copies of the same operands when split-K applies to
+ * neither (a panel of a tall problem may have few enough tiles to be split where the whole problem
+ * is not; both results pass the same error gates).
  *   A_host M x K (lda >= K), B_host K x N (ldb >= N), C_host M x N (ldc >= N), all FP32 HOST.
  * Errors: INVALID_ARG, ALLOC_FAILED, CUDA_ERROR, DEVICE_TIMEOUT. */
 int sgemm_cube_host(sgemm_cube_handle h, int M, int N, int K,

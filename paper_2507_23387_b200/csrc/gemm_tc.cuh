@@ -86,6 +86,16 @@ struct TcGemmParams {
   const float* B32;
   long long ldb32;
   float scale;          // 2^s
+  // Split-K (not FUSED, NTERMS == 3): the k range is cut into `ksplit` slices of `kslice_blocks`
+  // stages (a multiple of kchunk_blocks); unit u = slice * tiles + tile writes its hi*hi sums to
+  // Phh + slice * pstride and, termwise, its raw correction sums to Px + slice * pstride (both
+  // M x ldp); a reduction kernel forms C.  ksplit == 1: the kernel writes C itself.
+  int ksplit;
+  int kslice_blocks;
+  float* Phh;
+  float* Px;
+  long long pstride;
+  long long ldp;
 };
 
 template <int NTERMS, bool PAIR = false>
@@ -318,8 +328,16 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA0, const __grid_constant__
     if (PAIR) tm = tm * 2 + (int)cta_rank;
   };
   const int num_kb = (p.K + BK - 1) / BK;                      // pipeline stages per tile
+  const int ksplit = FUSED ? 1 : p.ksplit;
+  const int num_units = num_tiles * ksplit;
+  // Work unit -> tile coordinates and its range of stages [kb0, kb1).
+  auto unit_rc = [&](int unit, int& tm, int& tn, int& kb0, int& kb1, int& slice) {
+    slice = unit / num_tiles;
+    tile_rc(unit - slice * num_tiles, tm, tn);
+    kb0 = (ksplit > 1) ? slice * p.kslice_blocks : 0;
+    kb1 = (ksplit > 1) ? min(num_kb, kb0 + p.kslice_blocks) : num_kb;
+  };
   const int chunk = p.kchunk_blocks;                           // stages per k-block g
-  const int num_chunks = (num_kb + chunk - 1) / chunk;
 
   // Register budget when FUSED (512 threads x 128 registers): the accumulate warps hold a
   // 128 x 256 FP32 tile in registers, so warpgroups 2-3 hand registers over to warpgroups 0-1
@@ -348,10 +366,11 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA0, const __grid_constant__
       if (!PAIR || leader) mbar_arrive(&tempty_bar[r]);
       else mbar_arrive_cluster(mapa_u32(smem_u32(&tempty_bar[r]), 0));
     };
-    for (int tile = first_tile; tile < num_tiles && ok; tile += tile_stride) {
-      int tm, tn;
-      tile_rc(tile, tm, tn);
-      for (int c = 0; c < num_chunks && ok; ++c, ++gchunk) {
+    for (int unit = first_tile; unit < num_units && ok; unit += tile_stride) {
+      int tm, tn, kb0, kb1, slice;
+      unit_rc(unit, tm, tn, kb0, kb1, slice);
+      const int unit_chunks = (kb1 - kb0 + chunk - 1) / chunk;
+      for (int c = 0; c < unit_chunks && ok; ++c, ++gchunk) {
         const int r_main = (NTERMS == 1) ? (int)(gchunk & 1) : 0;
         const bool with_x = (NTERMS == 3) && (p.order == 1);
         {
@@ -399,8 +418,64 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA0, const __grid_constant__
       SGC_T0();
       const int row = tm * kBM + quarter * 32 + lane;
       const int col_base = tn * kBN + half * 128;
+      // Store the 128 values of this thread's row segment to a row-major matrix.  Vector path:
+      // storing straight from registers would write 16 bytes per row per instruction; instead
+      // 32 x 32 blocks go through a per-warp staging buffer (16-byte chunks XOR-swizzled by row:
+      // conflict-free both ways) and leave as 128-byte row segments, four rows per store.
+      auto store_tile = [&](float* base, long long ld, bool vec, int accumulate) {
+        if (vec) {
+          const uint32_t stg = smem_u32(store_staging + warp * 4096);
+          const int row0 = tm * kBM + quarter * 32;
+#pragma unroll
+          for (int g = 0; g < 4; ++g) {
+#pragma unroll
+            for (int q = 0; q < 8; ++q)
+              asm volatile("st.shared.v4.f32 [%0], {%1, %2, %3, %4};" ::"r"(
+                               stg + lane * 128 + ((q ^ (lane & 7)) << 4)),
+                           "f"(S[g * 32 + 4 * q]), "f"(S[g * 32 + 4 * q + 1]), "f"(S[g * 32 + 4 * q + 2]),
+                           "f"(S[g * 32 + 4 * q + 3])
+                           : "memory");
+            __syncwarp();
+            const int q = lane & 7;
+            const int col = col_base + g * 32 + q * 4;
+#pragma unroll
+            for (int i = 0; i < 8; ++i) {
+              const int r = i * 4 + (lane >> 3);
+              float4 v;
+              asm volatile("ld.shared.v4.f32 {%0, %1, %2, %3}, [%4];"
+                           : "=f"(v.x), "=f"(v.y), "=f"(v.z), "=f"(v.w)
+                           : "r"(stg + r * 128 + ((q ^ (r & 7)) << 4))
+                           : "memory");
+              const int grow = row0 + r;
+              if (grow < p.M && col < p.N) {
+                float* dst = base + (long long)grow * ld + col;
+                if (col + 4 <= p.N) {
+                  if (accumulate) {
+                    const float4 old = *reinterpret_cast<const float4*>(dst);
+                    v.x = __fadd_rn(old.x, v.x); v.y = __fadd_rn(old.y, v.y);
+                    v.z = __fadd_rn(old.z, v.z); v.w = __fadd_rn(old.w, v.w);
+                  }
+                  *reinterpret_cast<float4*>(dst) = v;
+                } else {
+                  const float e[4] = {v.x, v.y, v.z, v.w};
+                  for (int j = 0; j < 4 && col + j < p.N; ++j)
+                    dst[j] = accumulate ? __fadd_rn(dst[j], e[j]) : e[j];
+                }
+              }
+            }
+            __syncwarp();
+          }
+        } else {
+#pragma unroll
+          for (int g = 0; g < 8; ++g)
+            store16(base, ld, p.M, p.N, row, col_base + g * 16, &S[g * 16], false, accumulate);
+        }
+      };
+      const bool split_out = (NTERMS == 3) && (ksplit > 1);
+      if (split_out) store_tile(p.Phh + (long long)slice * p.pstride, p.ldp, true, 0);
       if (NTERMS == 3 && p.order == 0) {
-        // Termwise: the correction stream meets the dominant stream once, here.
+        // Termwise: the correction stream meets the dominant stream once: here, or (split-K) in
+        // the reduction kernel, which gets the raw correction sums of this slice.
         if (!wait_tfull(1)) {
           ok = false;
           break;
@@ -412,67 +487,22 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA0, const __grid_constant__
           uint32_t v[GW];
           tmem_ld_cols(t_x + g * GW, v);
           tmem_ld_wait();
+          if (split_out) {
 #pragma unroll
-          for (int j = 0; j < GW; ++j)
-            S[g * GW + j] = __fadd_rn(S[g * GW + j], __fmul_rn(__uint_as_float(v[j]), p.inv_scale));
+            for (int j = 0; j < GW; ++j) S[g * GW + j] = __uint_as_float(v[j]);
+          } else {
+#pragma unroll
+            for (int j = 0; j < GW; ++j)
+              S[g * GW + j] = __fadd_rn(S[g * GW + j], __fmul_rn(__uint_as_float(v[j]), p.inv_scale));
+          }
         }
         tc_fence_before_sync();
         __syncwarp();
         if (lane == 0) arrive_tempty(1);
         drains[1]++;
+        if (split_out) store_tile(p.Px + (long long)slice * p.pstride, p.ldp, true, 0);
       }
-      if (vec_ok) {
-        // Each thread owns one row of the tile; storing straight from registers would write 16
-        // bytes per row per instruction.  Instead 32 x 32 blocks go through a per-warp staging
-        // buffer (16-byte chunks XOR-swizzled by row: conflict-free both ways) and leave as
-        // 128-byte row segments, four rows per store instruction.
-        const uint32_t stg = smem_u32(store_staging + warp * 4096);
-        const int row0 = tm * kBM + quarter * 32;
-#pragma unroll
-        for (int g = 0; g < 4; ++g) {
-#pragma unroll
-          for (int q = 0; q < 8; ++q)
-            asm volatile("st.shared.v4.f32 [%0], {%1, %2, %3, %4};" ::"r"(
-                             stg + lane * 128 + ((q ^ (lane & 7)) << 4)),
-                         "f"(S[g * 32 + 4 * q]), "f"(S[g * 32 + 4 * q + 1]), "f"(S[g * 32 + 4 * q + 2]),
-                         "f"(S[g * 32 + 4 * q + 3])
-                         : "memory");
-          __syncwarp();
-          const int q = lane & 7;
-          const int col = col_base + g * 32 + q * 4;
-#pragma unroll
-          for (int i = 0; i < 8; ++i) {
-            const int r = i * 4 + (lane >> 3);
-            float4 v;
-            asm volatile("ld.shared.v4.f32 {%0, %1, %2, %3}, [%4];"
-                         : "=f"(v.x), "=f"(v.y), "=f"(v.z), "=f"(v.w)
-                         : "r"(stg + r * 128 + ((q ^ (r & 7)) << 4))
-                         : "memory");
-            const int grow = row0 + r;
-            if (grow < p.M && col < p.N) {
-              float* dst = p.D + (long long)grow * p.ldd + col;
-              if (col + 4 <= p.N) {
-                if (NTERMS == 1 && p.accumulate) {
-                  const float4 old = *reinterpret_cast<const float4*>(dst);
-                  v.x = __fadd_rn(old.x, v.x); v.y = __fadd_rn(old.y, v.y);
-                  v.z = __fadd_rn(old.z, v.z); v.w = __fadd_rn(old.w, v.w);
-                }
-                *reinterpret_cast<float4*>(dst) = v;
-              } else {
-                const float e[4] = {v.x, v.y, v.z, v.w};
-                for (int j = 0; j < 4 && col + j < p.N; ++j)
-                  dst[j] = (NTERMS == 1 && p.accumulate) ? __fadd_rn(dst[j], e[j]) : e[j];
-              }
-            }
-          }
-          __syncwarp();
-        }
-      } else {
-#pragma unroll
-        for (int g = 0; g < 8; ++g)
-          store16(p.D, p.ldd, p.M, p.N, row, col_base + g * 16, &S[g * 16], false,
-                  (NTERMS == 1) ? p.accumulate : 0);
-      }
+      if (!split_out) store_tile(p.D, p.ldd, vec_ok, (NTERMS == 1) ? p.accumulate : 0);
       SGC_TADD(8, blockIdx.x == 0 && threadIdx.x == 0);
     }
   } else if (warp == kMmaWarp) {
@@ -502,10 +532,13 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA0, const __grid_constant__
       uint32_t fills[2] = {0, 0};     // how many times each TMEM region has been handed over
       uint32_t gchunk = 0;            // running k-block counter (NTERMS == 1 region choice)
       bool ok = true;
-      for (int tile = first_tile; tile < num_tiles && ok; tile += tile_stride) {
-        for (int c = 0; c < num_chunks && ok; ++c, ++gchunk) {
-          const int kb_begin = c * chunk;
-          const int kb_end = min(num_kb, kb_begin + chunk);
+      for (int unit = first_tile; unit < num_units && ok; unit += tile_stride) {
+        int tm_, tn_, kb0, kb1, slice_;
+        unit_rc(unit, tm_, tn_, kb0, kb1, slice_);
+        const int unit_chunks = (kb1 - kb0 + chunk - 1) / chunk;
+        for (int c = 0; c < unit_chunks && ok; ++c, ++gchunk) {
+          const int kb_begin = kb0 + c * chunk;
+          const int kb_end = min(kb1, kb_begin + chunk);
           // Region(s) this k-block accumulates into, and which of them start from zero here.
           const int r_main = (NTERMS == 1) ? (int)(gchunk & 1) : 0;
           const bool x_fresh = (NTERMS == 3) && (p.order == 1 || c == 0);
@@ -590,7 +623,7 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA0, const __grid_constant__
           // Hand the finished region(s) to the accumulate warps.
           commit_both(&tfull_bar[r_main]);
           fills[r_main]++;
-          if (NTERMS == 3 && (p.order == 1 || c == num_chunks - 1)) {
+          if (NTERMS == 3 && (p.order == 1 || c == unit_chunks - 1)) {
             commit_both(&tfull_bar[1]);
             fills[1]++;
           }
@@ -611,11 +644,11 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA0, const __grid_constant__
         if (PAIR) tma_load_2d_pair(dst, map, x, y, bar);    // bytes counted on the leader's barrier
         else tma_load_2d(dst, map, x, y, bar);
       };
-      for (int tile = first_tile; tile < num_tiles && ok; tile += tile_stride) {
-        int tm, tn;
-        tile_rc(tile, tm, tn);
+      for (int unit = first_tile; unit < num_units && ok; unit += tile_stride) {
+        int tm, tn, kb0, kb1, slice;
+        unit_rc(unit, tm, tn, kb0, kb1, slice);
         const int n0 = tn * kBN + (PAIR ? (int)cta_rank * Cfg::BN_CTA : 0);   // this CTA's B columns
-        for (int kb = 0; kb < num_kb; ++kb, ++it) {
+        for (int kb = kb0; kb < kb1; ++kb, ++it) {
           const int s = it % STAGES;
           const uint32_t ph = (it / STAGES) & 1;
           if (!mbar_wait_bounded(&empty_bar[s], ph ^ 1, abort_flag, p.err, kErrProducerEmptyWait)) {

@@ -44,6 +44,9 @@ struct sgemm_cube_ctx {
   unsigned int* err_dev = nullptr;   // [0] error word; [4..8] scratch of sgemm_cube_exponent_window
   void* ws = nullptr;          // unfused path: FP16 words of A and B, D_hh, D_x
   size_t ws_bytes = 0;
+  void* part_ws = nullptr;     // split-K partial sums
+  size_t part_ws_bytes = 0;
+  int split_k = 1;             // 1: split the k range of few-tile problems over idle SMs; 0: never
   void* host_ws = nullptr;     // host-buffer path: device copies of A, B, C
   size_t host_ws_bytes = 0;
   long long launches = 0;
@@ -154,7 +157,7 @@ int launch_tc_kernel(sgemm_cube_ctx* h, int M, int N, const CUtensorMap& tmA0, c
     const int units = ((M + 2 * sgc::kBM - 1) / (2 * sgc::kBM)) * tiles_n;
     cfg.gridDim = dim3(2 * (units < cached ? units : cached), 1, 1);
   } else {
-    const int units = ((M + sgc::kBM - 1) / sgc::kBM) * tiles_n;
+    const int units = ((M + sgc::kBM - 1) / sgc::kBM) * tiles_n * (p.ksplit > 1 ? p.ksplit : 1);
     cfg.gridDim = dim3(units < h->sm_count ? units : h->sm_count, 1, 1);
   }
   h->launches++;
@@ -222,7 +225,48 @@ int launch_tc_gemm(sgemm_cube_ctx* h, int M, int N, int K, const uint16_t* Ahi, 
   p.inv_scale = inv_scale;
   p.err = h->err_dev;
   p.A32 = nullptr; p.lda32 = 0; p.B32 = nullptr; p.ldb32 = 0; p.scale = 1.f;
-  return use_pair(h, M, N) ? launch_tc_kernel<NTERMS, false, true>(h, M, N, tmA0, tmA1, tmB0, tmB1, p, st)
+  p.ksplit = 1; p.kslice_blocks = 0; p.Phh = nullptr; p.Px = nullptr; p.pstride = 0; p.ldp = 0;
+  // Split-K: when the tiles would leave more than half of the SMs idle and k is long, cut the k
+  // range into slices (whole k-blocks) so that tiles x slices fills the machine; a reduction
+  // kernel adds the slices' sums.
+  const bool pair = use_pair(h, M, N);
+  if (NTERMS == 3 && h->split_k && !pair) {
+    const int tiles = ((M + sgc::kBM - 1) / sgc::kBM) * ((N + sgc::kBN - 1) / sgc::kBN);
+    const int num_kb = (K + Cfg::BK - 1) / Cfg::BK;
+    const int chunks = (num_kb + p.kchunk_blocks - 1) / p.kchunk_blocks;
+    int want = h->sm_count / tiles;
+    if (want > 16) want = 16;
+    if (want > K / 1024) want = K / 1024;       // a slice shorter than 1024 costs more than it saves
+    if (want >= 2 && chunks >= 2 * want) {
+      const int chunks_per_slice = (chunks + want - 1) / want;
+      const int slices = (chunks + chunks_per_slice - 1) / chunks_per_slice;
+      const size_t ldp = round_up((size_t)N, 4);
+      const size_t pstride = round_up((size_t)M * ldp, 64);
+      const size_t need = (size_t)slices * pstride * 4 * (order == SGEMM_CUBE_TERMWISE ? 2 : 1);
+      if (slices >= 2 && grow(&h->part_ws, &h->part_ws_bytes, need) == SGEMM_CUBE_OK) {
+        p.ksplit = slices;
+        p.kslice_blocks = chunks_per_slice * p.kchunk_blocks;
+        p.Phh = static_cast<float*>(h->part_ws);
+        p.Px = p.Phh + (size_t)slices * pstride;
+        p.pstride = (long long)pstride;
+        p.ldp = (long long)ldp;
+      }
+    }
+  }
+  if (p.ksplit > 1) {
+    rc = launch_tc_kernel<NTERMS, false, false>(h, M, N, tmA0, tmA1, tmB0, tmB1, p, st);
+    if (rc) return rc;
+    const long long total = (long long)M * N;
+    long long blocks = (total + 255) / 256;
+    const long long cap = (long long)h->sm_count * 16;
+    if (blocks > cap) blocks = cap;
+    sgc::splitk_reduce_kernel<<<(unsigned)blocks, 256, 0, st>>>(M, N, p.ksplit, p.Phh, p.Px, p.pstride, p.ldp,
+                                                                 D, ldd, inv_scale,
+                                                                 order == SGEMM_CUBE_TERMWISE ? 1 : 0);
+    h->launches++;
+    return cudaGetLastError() == cudaSuccess ? SGEMM_CUBE_OK : SGEMM_CUBE_CUDA_ERROR;
+  }
+  return pair ? launch_tc_kernel<NTERMS, false, true>(h, M, N, tmA0, tmA1, tmB0, tmB1, p, st)
                            : launch_tc_kernel<NTERMS, false, false>(h, M, N, tmA0, tmA1, tmB0, tmB1, p, st);
 }
 
@@ -244,6 +288,7 @@ int launch_fused(sgemm_cube_ctx* h, int M, int N, int K, const float* A, int64_t
   p.A32 = A; p.lda32 = lda;
   p.B32 = B; p.ldb32 = ldb;
   p.scale = ldexpf(1.0f, s);
+  p.ksplit = 1; p.kslice_blocks = 0; p.Phh = nullptr; p.Px = nullptr; p.pstride = 0; p.ldp = 0;
   CUtensorMap unused;
   memset(&unused, 0, sizeof(unused));
   return use_pair(h, M, N) ? launch_tc_kernel<3, true, true>(h, M, N, unused, unused, unused, unused, p, st)
@@ -364,6 +409,7 @@ int sgemm_cube_destroy(sgemm_cube_handle h) {
     rc = SGEMM_CUBE_DEVICE_TIMEOUT;
   if (h->ws) cudaFree(h->ws);
   if (h->host_ws) cudaFree(h->host_ws);
+  if (h->part_ws) cudaFree(h->part_ws);
   if (h->ev0) cudaEventDestroy(h->ev0);
   if (h->ev1) cudaEventDestroy(h->ev1);
   if (h->s_in) cudaStreamDestroy(h->s_in);
@@ -385,6 +431,11 @@ int sgemm_cube_set_option(sgemm_cube_handle h, int option, int64_t value) {
   if (option == SGEMM_CUBE_OPT_CTA_PAIR) {
     if (value < 0 || value > 2) return SGEMM_CUBE_INVALID_ARG;
     h->cta_pair = (int)value;
+    return SGEMM_CUBE_OK;
+  }
+  if (option == SGEMM_CUBE_OPT_SPLIT_K) {
+    if (value != 0 && value != 1) return SGEMM_CUBE_INVALID_ARG;
+    h->split_k = (int)value;
     return SGEMM_CUBE_OK;
   }
   if (option == SGEMM_CUBE_OPT_STRATEGY) {

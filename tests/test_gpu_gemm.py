@@ -158,17 +158,43 @@ def test_cta_pair_mode_is_bit_identical(handle, path, order):
     # tcgen05.mma.cta_group::2 (two CTAs per 256 x 256 tile) against one CTA per 128 x 256 tile.
     res = {}
     try:
+        handle.sgemm_cube_set_option(binding.OPT_SPLIT_K, 0)     # split-K applies to single CTAs only
         for pair in (0, 1):
             handle.sgemm_cube_set_option(binding.OPT_CTA_PAIR, pair)
             res[pair] = [run(handle, path, padded_dev(A, 4), padded_dev(B, 4), 11, order)
                          for (A, B) in (inputs.make_pair("normal", 6, M, N, K)
                                         for (M, N, K) in [(512, 768, 520), (129, 300, 97), (1024, 256, 2048)])]
     finally:
-        handle.sgemm_cube_set_option(binding.OPT_CTA_PAIR, 2)
+        handle.sgemm_cube_set_option(binding.OPT_CTA_PAIR, 0)
+        handle.sgemm_cube_set_option(binding.OPT_SPLIT_K, 1)
     for a, b in zip(res[0], res[1]):
         assert np.array_equal(a, b)
     A, B = inputs.make_pair("normal", 6, 129, 300, 97)
     gates(res[1][1], A, B, 11, order, label="pair %s" % path)
+
+
+@pytest.mark.parametrize("path,order", [("two_phase", T), ("two_phase", E), ("presplit", T)])
+@pytest.mark.parametrize("shape", [(256, 256, 4096), (300, 520, 3000), (128, 256, 513), (1024, 1024, 8192)])
+def test_split_k_on_few_tile_shapes(handle, path, order, shape):
+    # Few tiles and a long k: the k range is cut into slices that run on otherwise idle SMs and a
+    # reduction kernel adds the slices' sums.  Same gates; and switching it off must still pass.
+    M, N, K = shape
+    A, B = inputs.make_pair("normal", 13, M, N, K)
+    Ad, Bd = padded_dev(A, 4), padded_dev(B, 4)
+    res = {}
+    try:
+        for on in (1, 0):
+            handle.sgemm_cube_set_option(binding.OPT_SPLIT_K, on)
+            res[on] = run(handle, path, Ad, Bd, 11, order)
+            gates(res[on], A, B, 11, order, label="split-k %d %s %s" % (on, path, shape))
+    finally:
+        handle.sgemm_cube_set_option(binding.OPT_SPLIT_K, 1)
+    # exact inputs: identical whatever the slicing
+    rng = np.random.default_rng(3)
+    Ai = rng.integers(-8, 9, size=(M, K)).astype(np.float32)
+    Bi = rng.integers(-8, 9, size=(K, N)).astype(np.float32)
+    Ci = run(handle, path, padded_dev(Ai, 4), padded_dev(Bi, 4), 11, order)
+    assert np.array_equal(Ci, (Ai.astype(np.int64) @ Bi.astype(np.int64)).astype(np.float32))
 
 
 def test_k_block_option_changes_bracketing_not_validity(handle):
@@ -272,7 +298,11 @@ def test_config5_large_shapes_sampled_rows(handle, shape):
     perm = torch.randperm(256, device="cuda:0", generator=torch.Generator("cuda:0").manual_seed(0))
     A2 = A[:256][perm].contiguous()
     C2 = torch.empty((256, N), device="cuda:0")
-    handle.sgemm_cube(A2, B, C2, 11, T)
+    handle.sgemm_cube_set_option(binding.OPT_SPLIT_K, 0)      # same k bracketing as the full problem
+    try:
+        handle.sgemm_cube(A2, B, C2, 11, T)
+    finally:
+        handle.sgemm_cube_set_option(binding.OPT_SPLIT_K, 1)
     assert torch.equal(C2, C[:256][perm])
 
 

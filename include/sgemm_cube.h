@@ -74,9 +74,9 @@ enum {
    * tcgen05.mma.cta_group::2 (256 x 256 tile per pair, each CTA loading half of the B tile);
    * 0 (default): one CTA per 128 x 256 tile; 2: pairs when the problem has at least four waves
    * of pair tiles.  Same arithmetic, bit-identical results either way as long as split-K (below,
-   * single CTAs only) does not apply.  (Pairs halve the B-tile
-   * traffic and are the faster mode for k-blocks of 512 and more; at the default k-block of 256
-   * the more frequent TMEM drains cost them more than they save.) */
+   * single CTAs only) does not apply.  (Pairs halve the B-tile traffic and are the faster mode
+   * for k-blocks of 512 and more; at the default k-block of 128 the more frequent TMEM drains
+   * cost them more than they save.) */
   SGEMM_CUBE_OPT_CTA_PAIR = 2,
   /* How sgemm_cube computes (same arithmetic; same bracketing and bit-identical results except
    * where split-K, which only the two-phase strategy uses, re-brackets the k-block sums):

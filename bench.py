@@ -4,8 +4,10 @@
     python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference]
 
 One "step" is one pass of the whole hot path over one batch of synthetic input: a single call of
-the fused `sgemm_cube` entry point (operand split, three FP16 tensor-core products and the FP32
-reconstruction in one kernel) on M = N = K = 8192 FP32 matrices whose entries are
+the `sgemm_cube` entry point with its default options (operand split, three FP16 tensor-core
+products and the FP32 reconstruction; at this size the library splits both operands once with the
+split kernel and forms the products in one tensor-core kernel: three launches per step) on
+M = N = K = 8192 FP32 matrices whose entries are
 (+/-) u * 2^e, u uniform in [1, 2), e a uniform integer in [-10, 10], with s = 11 and termwise
 accumulation.  The metric is FP32-equivalent TFLOP/s = 2 M N K / t.
 

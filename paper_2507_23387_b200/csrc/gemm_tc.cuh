@@ -98,9 +98,14 @@ struct TcGemmParams {
   long long ldp;
 };
 
-template <int NTERMS, bool PAIR = false>
+#ifndef SGC_BK3
+#define SGC_BK3 32
+#endif
+template <int NTERMS, bool PAIR = false, bool FUSED = false>
 struct TcCfg {
-  static constexpr int BK = (NTERMS == 1) ? 64 : 32;      // k per pipeline stage
+  // k per pipeline stage: 64 for one product; for three products 32 when the converter warps fill
+  // the stages, SGC_BK3 (32 or 16) when TMA does
+  static constexpr int BK = (NTERMS == 1) ? 64 : (FUSED ? 32 : SGC_BK3);
   static constexpr int BN_CTA = PAIR ? kBN / 2 : kBN;     // B columns held by one CTA
   static constexpr int A_ROW_BYTES = BK * 2;              // 128 or 64: also the swizzle span of A
   static constexpr uint32_t A_TILE = kBM * BK * 2;        // one FP16 A tile
@@ -250,7 +255,7 @@ __global__ void __launch_bounds__(FUSED ? kFusedThreads : kTcThreads, 1)
 tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA0, const __grid_constant__ CUtensorMap tmA1,
                const __grid_constant__ CUtensorMap tmB0, const __grid_constant__ CUtensorMap tmB1,
                const TcGemmParams p) {
-  using Cfg = TcCfg<NTERMS, PAIR>;
+  using Cfg = TcCfg<NTERMS, PAIR, FUSED>;
   constexpr int BK = Cfg::BK;
   constexpr int STAGES = Cfg::STAGES;
   // PAIR: the kernel runs as clusters of two CTAs driving tcgen05.mma.cta_group::2.  The pair owns
@@ -524,7 +529,8 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA0, const __grid_constant__
         return PAIR ? mbar_wait_bounded_cluster(bar, parity, abort_flag, p.err, code)
                     : mbar_wait_bounded(bar, parity, abort_flag, p.err, code);
       };
-      constexpr uint64_t a_swz = (Cfg::A_ROW_BYTES == 128) ? kSwizzle128 : kSwizzle64;
+      constexpr uint64_t a_swz = (Cfg::A_ROW_BYTES == 128) ? kSwizzle128
+                                 : (Cfg::A_ROW_BYTES == 64) ? kSwizzle64 : kSwizzle32;
       constexpr uint32_t a_sbo = 8 * Cfg::A_ROW_BYTES;     // 8 rows of the swizzle atom
       constexpr uint32_t b_lbo = BK * 128;                 // next 64-column atom of B
       constexpr uint32_t b_sbo = 1024;                     // next 8 k-rows inside an atom

@@ -126,7 +126,7 @@ __device__ __forceinline__ void tmem_dealloc(uint32_t taddr, uint32_t ncols) {
 // Shared-memory matrix descriptor (64 bit): start address >> 4 in bits [0,14), leading byte
 // offset >> 4 in [16,30), stride byte offset >> 4 in [32,46), descriptor version 1 in [46,48),
 // swizzle mode in [61,64) (2 = 128-byte, 4 = 64-byte, 6 = 32-byte, 0 = none).
-constexpr uint64_t kSwizzle128 = 2, kSwizzle64 = 4;
+constexpr uint64_t kSwizzle128 = 2, kSwizzle64 = 4, kSwizzle32 = 6;
 __device__ __forceinline__ uint64_t umma_smem_desc(uint32_t smem_addr, uint32_t lbo_bytes,
                                                    uint32_t sbo_bytes, uint64_t swizzle) {
   return (uint64_t)((smem_addr & 0x3FFFFu) >> 4) | ((uint64_t)((lbo_bytes >> 4) & 0x3FFFu) << 16) |

@@ -104,10 +104,10 @@ int set_kernel_attrs(sgemm_cube_ctx* h) {
   const cudaFuncAttribute attr = cudaFuncAttributeMaxDynamicSharedMemorySize;
   if (cudaFuncSetAttribute(sgc::tc_gemm_kernel<1, false, false>, attr, (int)sgc::TcCfg<1, false>::SMEM_BYTES) != cudaSuccess ||
       cudaFuncSetAttribute(sgc::tc_gemm_kernel<3, false, false>, attr, (int)sgc::TcCfg<3, false>::SMEM_BYTES) != cudaSuccess ||
-      cudaFuncSetAttribute(sgc::tc_gemm_kernel<3, true, false>, attr, (int)sgc::TcCfg<3, false>::SMEM_BYTES) != cudaSuccess ||
+      cudaFuncSetAttribute(sgc::tc_gemm_kernel<3, true, false>, attr, (int)sgc::TcCfg<3, false, true>::SMEM_BYTES) != cudaSuccess ||
       cudaFuncSetAttribute(sgc::tc_gemm_kernel<1, false, true>, attr, (int)sgc::TcCfg<1, true>::SMEM_BYTES) != cudaSuccess ||
       cudaFuncSetAttribute(sgc::tc_gemm_kernel<3, false, true>, attr, (int)sgc::TcCfg<3, true>::SMEM_BYTES) != cudaSuccess ||
-      cudaFuncSetAttribute(sgc::tc_gemm_kernel<3, true, true>, attr, (int)sgc::TcCfg<3, true>::SMEM_BYTES) != cudaSuccess) {
+      cudaFuncSetAttribute(sgc::tc_gemm_kernel<3, true, true>, attr, (int)sgc::TcCfg<3, true, true>::SMEM_BYTES) != cudaSuccess) {
     cudaGetLastError();
     return SGEMM_CUBE_CUDA_ERROR;
   }
@@ -128,7 +128,7 @@ template <int NTERMS, bool FUSED, bool PAIR>
 int launch_tc_kernel(sgemm_cube_ctx* h, int M, int N, const CUtensorMap& tmA0, const CUtensorMap& tmA1,
                      const CUtensorMap& tmB0, const CUtensorMap& tmB1, const sgc::TcGemmParams& p,
                      cudaStream_t st) {
-  using Cfg = sgc::TcCfg<NTERMS, PAIR>;
+  using Cfg = sgc::TcCfg<NTERMS, PAIR, FUSED>;
   auto kernel = sgc::tc_gemm_kernel<NTERMS, FUSED, PAIR>;
   cudaLaunchConfig_t cfg;
   memset(&cfg, 0, sizeof(cfg));
@@ -199,7 +199,8 @@ int launch_tc_gemm(sgemm_cube_ctx* h, int M, int N, int K, const uint16_t* Ahi, 
   if (rc) return rc;
   CUtensorMap tmA0, tmA1, tmB0, tmB1;
   const CUtensorMapSwizzle a_swz =
-      (Cfg::A_ROW_BYTES == 128) ? CU_TENSOR_MAP_SWIZZLE_128B : CU_TENSOR_MAP_SWIZZLE_64B;
+      (Cfg::A_ROW_BYTES == 128) ? CU_TENSOR_MAP_SWIZZLE_128B
+      : (Cfg::A_ROW_BYTES == 64) ? CU_TENSOR_MAP_SWIZZLE_64B : CU_TENSOR_MAP_SWIZZLE_32B;
   rc = make_map(h, &tmA0, CU_TENSOR_MAP_DATA_TYPE_FLOAT16, 2, Ahi, K, M, lda16, Cfg::BK, sgc::kBM, a_swz);
   if (rc) return rc;
   rc = make_map(h, &tmB0, CU_TENSOR_MAP_DATA_TYPE_FLOAT16, 2, Bhi, N, K, ldb16, 64, Cfg::BK,
@@ -272,7 +273,7 @@ int launch_tc_gemm(sgemm_cube_ctx* h, int M, int N, int K, const uint16_t* Ahi, 
 
 int launch_fused(sgemm_cube_ctx* h, int M, int N, int K, const float* A, int64_t lda, const float* B,
                  int64_t ldb, float* C, int64_t ldc, int s, int order, cudaStream_t st) {
-  using Cfg = sgc::TcCfg<3, false>;
+  using Cfg = sgc::TcCfg<3, false, true>;
   int rc = set_kernel_attrs(h);
   if (rc) return rc;
   sgc::TcGemmParams p;

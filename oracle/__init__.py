@@ -49,6 +49,9 @@ def _load():
         lib.oracle_sgemm_cube.argtypes = [i64, i64, i64, vp, i64, vp, i64, vp, i64, c_int, c_int,
                                           i64, vp, i64]
         lib.oracle_sgemm_cube.restype = c_int
+        lib.oracle_sgemm_cube_four_term.argtypes = [i64, i64, i64, vp, i64, vp, i64, vp, i64,
+                                                    c_int, i64]
+        lib.oracle_sgemm_cube_four_term.restype = c_int
         lib.oracle_dgemm_ref.argtypes = [i64, i64, i64, vp, i64, vp, i64, vp, vp]
         lib.oracle_dgemm_ref.restype = None
         lib.oracle_sgemm_f32.argtypes = [i64, i64, i64, vp, i64, vp, i64, vp, i64]
@@ -121,6 +124,25 @@ def sgemm_cube(A, B, s=11, order=TERMWISE, kb=64, return_hgemm=False):
     if rc != 0:
         raise ValueError("oracle_sgemm_cube: invalid argument")
     return (C, H) if return_hgemm else C
+
+
+def sgemm_cube_four_term(A, B, s=11, kb=64):
+    """C = hi_A hi_B + 2^-s (lo_A hi_B + hi_A lo_B) + 2^-2s lo_A lo_B, termwise, k-blocks of kb
+    (Eq. recover_eqn with the low-low product of Eq. ll_bound kept)."""
+    lib = _load()
+    A, B = _f32_2d(A), _f32_2d(B)
+    M, K = A.shape
+    K2, N = B.shape
+    if K != K2:
+        raise ValueError("inner dimensions differ")
+    C = np.empty((M, N), dtype=np.float32)
+    kb = int(kb) if kb else max(K, 1)
+    rc = lib.oracle_sgemm_cube_four_term(M, N, K, A.ctypes.data, A.strides[0] // 4,
+                                         B.ctypes.data, B.strides[0] // 4, C.ctypes.data, N,
+                                         int(s), kb)
+    if rc != 0:
+        raise ValueError("oracle_sgemm_cube_four_term: invalid argument")
+    return C
 
 
 def dgemm_ref(A, B, with_abs=True):

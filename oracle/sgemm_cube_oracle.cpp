@@ -217,6 +217,66 @@ int oracle_sgemm_cube(int64_t M, int64_t N, int64_t K,
   return 0;
 }
 
+// Four-term variant: the full expansion of (hi_A + lo_A/s_f)(hi_B + lo_B/s_f), i.e. Eq.
+// recover_eqn with the low-low product that Eq. ll_bound bounds kept instead of dropped:
+//   C = hi_A hi_B + 2^-s (lo_A hi_B + hi_A lo_B) + 2^-2s lo_A lo_B.
+// Termwise only: each of the four streams is summed in k-blocks of kb as in oracle_sgemm_cube; the
+// small terms are combined among themselves, smallest first, and meet the dominant stream once:
+//   C = S_hh + ((S_lh + S_hl) 2^-s + S_ll 2^-2s).
+int oracle_sgemm_cube_four_term(int64_t M, int64_t N, int64_t K,
+                                const float* A, int64_t lda, const float* B, int64_t ldb,
+                                float* C, int64_t ldc, int s, int64_t kb) {
+  if (M < 0 || N < 0 || K < 0 || kb <= 0 || s < 0 || s > 24) return 1;
+  std::vector<float> Bh((size_t)K * N), Bl((size_t)K * N);
+#pragma omp parallel for schedule(static)
+  for (int64_t k = 0; k < K; ++k)
+    for (int64_t j = 0; j < N; ++j) {
+      uint16_t h, l;
+      split1(B[k * ldb + j], s, &h, &l);
+      Bh[(size_t)k * N + j] = bits_f32(f16_to_f32(h));
+      Bl[(size_t)k * N + j] = bits_f32(f16_to_f32(l));
+    }
+  const float inv_sf = std::ldexp(1.0f, -s);
+  const float inv_sf2 = std::ldexp(1.0f, -2 * s);
+#pragma omp parallel
+  {
+    std::vector<float> P(4 * (size_t)N), S(4 * (size_t)N);   // hh, lh, hl, ll
+    std::vector<float> Ah(K), Al(K);
+#pragma omp for schedule(dynamic, 1)
+    for (int64_t i = 0; i < M; ++i) {
+      for (int64_t k = 0; k < K; ++k) {
+        uint16_t h, l;
+        split1(A[i * lda + k], s, &h, &l);
+        Ah[k] = bits_f32(f16_to_f32(h));
+        Al[k] = bits_f32(f16_to_f32(l));
+      }
+      for (size_t t = 0; t < S.size(); ++t) S[t] = 0.f;
+      for (int64_t k0 = 0; k0 < K; k0 += kb) {
+        const int64_t k1 = (k0 + kb < K) ? k0 + kb : K;
+        for (size_t t = 0; t < P.size(); ++t) P[t] = 0.f;
+        for (int64_t k = k0; k < k1; ++k) {
+          const float ah = Ah[k], al = Al[k];
+          const float* bh = &Bh[(size_t)k * N];
+          const float* bl = &Bl[(size_t)k * N];
+          for (int64_t j = 0; j < N; ++j) {
+            P[j] = P[j] + ah * bh[j];
+            P[N + j] = P[N + j] + al * bh[j];
+            P[2 * N + j] = P[2 * N + j] + ah * bl[j];
+            P[3 * N + j] = P[3 * N + j] + al * bl[j];      // FP16 x FP16: exact in FP32
+          }
+        }
+        for (size_t t = 0; t < S.size(); ++t) S[t] = S[t] + P[t];
+      }
+      for (int64_t j = 0; j < N; ++j) {
+        const float cross = S[N + j] + S[2 * N + j];
+        const float small = cross * inv_sf + S[3 * N + j] * inv_sf2;
+        C[i * ldc + j] = S[j] + small;
+      }
+    }
+  }
+  return 0;
+}
+
 // FP64 reference C64 = A B and the matrix |A||B|, both accumulated in double.
 void oracle_dgemm_ref(int64_t M, int64_t N, int64_t K,
                       const float* A, int64_t lda, const float* B, int64_t ldb,

@@ -209,6 +209,23 @@ int sgemm_cube_host(sgemm_cube_handle h, int M, int N, int K,
                     float* C_host, int64_t ldc,
                     int scale_exp, int accumulation_order, void* stream);
 
+/* Four-term variant: the low-low product that SGEMM-cube drops (paper Sec. 4.3, bounded by
+ * Eq. ll_bound) is kept, i.e. the full expansion of (hi_A + lo_A 2^-s)(hi_B + lo_B 2^-s):
+ *   C = hi_A hi_B + 2^-s (lo_A hi_B + hi_A lo_B) + 2^-2s lo_A lo_B.
+ * It exists to measure what dropping that term costs; it is not part of the paper's method.
+ * Termwise only: each stream is summed in k-blocks (SGEMM_CUBE_OPT_TERMWISE_K_BLOCK) and
+ *   C = S_hh + (2^-s S_x + 2^-2s S_ll),
+ * the small terms combined first.  Runs as: two split launches, one FP16 GEMM pass lo_A lo_B into
+ * the handle's workspace, the three-product kernel writing its raw sums, one reduction kernel.
+ * Arguments, layouts and alignment-free inputs as sgemm_cube_unfused.  Workspace:
+ * 4 bytes x (M K + K N) + 12 bytes x M N, rounded up, grown with cudaMalloc on first use.
+ * Errors: INVALID_ARG, ALLOC_FAILED, CUDA_ERROR. */
+int sgemm_cube_four_term(sgemm_cube_handle h, int M, int N, int K,
+                         const float* A_dev, int64_t lda,
+                         const float* B_dev, int64_t ldb,
+                         float* C_dev, int64_t ldc,
+                         int scale_exp, void* stream);
+
 /* Exponent window of a matrix's FP16 high words (paper Sec. 4.2: e_min and e_max of
  * Eq. sf_bounds are the smallest and largest unbiased exponents E' - 15 of the finite high
  * components).  One pass over X on the device; the call synchronises `stream` and writes to HOST

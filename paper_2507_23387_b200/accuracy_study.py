@@ -9,9 +9,11 @@ Eq. err, mean over seeds):
                    and an FP32 GEMM                                  (Fig. scaling_bit_error)
   size sweep       error against m = n, against k, and against all three, at offset exponent 0
                                                                       (Fig. mkn_error)
+  dropped term     three-term SGEMM-cube against the four-term variant that keeps lo_A lo_B
+                   (the term Eq. ll_bound bounds), against k
 
 Everything runs through the library's C ABI (`sgemm_cube`, `sgemm_cube_split`,
-`sgemm_cube_hgemm`); the FP64 reference and the FP32 baseline are torch matmuls on the device.
+`sgemm_cube_hgemm`, `sgemm_cube_four_term`); the FP64 reference and the FP32 baseline are torch matmuls on the device.
 Run as a script for a markdown report:
 
     python -m paper_2507_23387_b200.accuracy_study [--size 1024] [--seeds 5] [--quick]
@@ -67,6 +69,8 @@ def measure(h, A, B, scale_exps=(0, 6, 11, 12)):
         for name, order in (("termwise", binding.TERMWISE), ("elementwise", binding.ELEMENTWISE)):
             h.sgemm_cube(A, B, C, s, order)
             out["%s_s%d" % (name, s)] = frobenius_rel_err(C, C64)
+        h.sgemm_cube_four_term(A, B, C, s)
+        out["four_term_s%d" % s] = frobenius_rel_err(C, C64)
     status, detail = h.sgemm_cube_check()
     if status != 0:
         raise RuntimeError("device error %s" % hex(detail))
@@ -111,6 +115,33 @@ def size_sweep(h, shapes, seeds=5, scale_exp=12, device="cuda:0"):
     return rows
 
 
+def dropped_term_sweep(h, ks=(8, 32, 128, 512, 2048, 8192), mn=1024, seeds=5, scale_exp=11,
+                       device="cuda:0"):
+    """Three-term against four-term error over the inner dimension (symmetric U[-1, 1) inputs):
+    Frobenius error as elsewhere, plus the largest componentwise error
+    max |C - C64| / (|A||B|) (the quantity Eq. main_bound and Eq. ll_bound are stated in)."""
+    rows = []
+    C = torch.empty((mn, mn), device=device)
+    for K in ks:
+        r = {"k": K, "three_term_frob": 0.0, "four_term_frob": 0.0, "three_term_cw": 0.0,
+             "four_term_cw": 0.0}
+        for seed in range(seeds):
+            A = torch.from_numpy(inputs.uniform_range(seed, (mn, K), 0, False, stream=0)).to(device)
+            B = torch.from_numpy(inputs.uniform_range(seed, (K, mn), 0, False, stream=1)).to(device)
+            C64 = _reference(A, B)
+            AB = A.double().abs() @ B.double().abs()
+            for name, call in (("three_term", lambda: h.sgemm_cube(A, B, C, scale_exp, binding.TERMWISE)),
+                               ("four_term", lambda: h.sgemm_cube_four_term(A, B, C, scale_exp))):
+                call()
+                r[name + "_frob"] += frobenius_rel_err(C, C64) / seeds
+                r[name + "_cw"] = max(r[name + "_cw"], float(((C.double() - C64).abs() / AB).max()))
+        rows.append(r)
+    status, detail = h.sgemm_cube_check()
+    if status != 0:
+        raise RuntimeError("device error %s" % hex(detail))
+    return rows
+
+
 def _table(rows, key, cols):
     lines = ["| %s | %s |" % (key, " | ".join(cols)), "|" + "---|" * (len(cols) + 1)]
     for r in rows:
@@ -137,7 +168,9 @@ def main():
     alls = [(n, n, n) for n in ((512, 2048) if args.quick else (512, 1024, 2048, 4096))]
     scol = ["fp16_hgemm", "fp32_gemm", "termwise_s12", "elementwise_s12"]
     res = {"symmetric": sym, "nonnegative": pos, "vs_mn": size_sweep(h, mn, args.seeds),
-           "vs_k": size_sweep(h, ks, args.seeds), "vs_all": size_sweep(h, alls, args.seeds)}
+           "vs_k": size_sweep(h, ks, args.seeds), "vs_all": size_sweep(h, alls, args.seeds),
+           "dropped_term": dropped_term_sweep(h, (8, 512) if args.quick else (8, 32, 128, 512, 2048, 8192),
+                                              seeds=args.seeds)}
     h.destroy()
     if args.json:
         print(json.dumps(res))
@@ -152,6 +185,9 @@ def main():
     print(_table(res["vs_k"], "shape", scol))
     print("\n## Relative error vs m = n = k\n")
     print(_table(res["vs_all"], "shape", scol))
+    print("\n## Three-term against four-term (low-low product kept), m = n = 1024, U[-1, 1), s_b = 11\n")
+    print(_table(res["dropped_term"], "k", ["three_term_frob", "four_term_frob", "three_term_cw",
+                                            "four_term_cw"]))
 
 
 if __name__ == "__main__":

@@ -20,6 +20,7 @@ STRATEGY_AUTO, STRATEGY_FUSED, STRATEGY_TWO_PHASE = 0, 1, 2
 
 EXPORTS = ["sgemm_cube_create", "sgemm_cube_destroy", "sgemm_cube_set_option", "sgemm_cube_split",
            "sgemm_cube", "sgemm_cube_unfused", "sgemm_cube_presplit", "sgemm_cube_hgemm",
+           "sgemm_cube_four_term",
            "sgemm_cube_host", "sgemm_cube_unfused_static", "sgemm_cube_check", "sgemm_cube_launch_count", "sgemm_cube_last_kernel_ms",
            "sgemm_cube_exponent_window", "sgemm_cube_choose_scale_exp",
            "sgemm_cube_status_string", "sgemm_cube_version"]
@@ -55,6 +56,7 @@ def load():
                                         i32, vp]
     lib.sgemm_cube_hgemm.argtypes = [vp, i32, i32, i32, vp, i64, vp, i64, vp, i64, i32, vp]
     lib.sgemm_cube_unfused_static.argtypes = [i32, i32, i32, vp, i64, vp, i64, vp, i64, i32, vp]
+    lib.sgemm_cube_four_term.argtypes = [vp, i32, i32, i32, vp, i64, vp, i64, vp, i64, i32, vp]
     lib.sgemm_cube_check.argtypes = [vp, vp, ctypes.POINTER(ctypes.c_uint32)]
     lib.sgemm_cube_last_kernel_ms.argtypes = [vp, ctypes.POINTER(ctypes.c_float)]
     lib.sgemm_cube_exponent_window.argtypes = [vp, i32, i32, vp, i64, ctypes.POINTER(i64), vp]
@@ -169,6 +171,16 @@ class Handle:
 
     def sgemm_cube_unfused(self, A, B, C, scale_exp=11, order=TERMWISE, stream=None):
         self._gemm(load().sgemm_cube_unfused, "sgemm_cube_unfused", A, B, C, scale_exp, order, stream)
+
+    def sgemm_cube_four_term(self, A, B, C, scale_exp=11, stream=None):
+        """The variant that keeps the low-low product (termwise only)."""
+        M, K = A.shape
+        K2, N = B.shape
+        assert K == K2 and C.shape == (M, N)
+        _check(load().sgemm_cube_four_term(self._h, M, N, K, _dev(A, torch.float32), _ld(A),
+                                           _dev(B, torch.float32), _ld(B), _dev(C, torch.float32),
+                                           _ld(C), scale_exp, _stream_ptr(stream)),
+               "sgemm_cube_four_term")
 
     def sgemm_cube_presplit(self, Ahi, Alo, Bhi, Blo, C, scale_exp=11, order=TERMWISE, stream=None):
         M, K = Ahi.shape

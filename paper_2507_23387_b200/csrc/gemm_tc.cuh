@@ -89,7 +89,9 @@ struct TcGemmParams {
   // Split-K (not FUSED, NTERMS == 3): the k range is cut into `ksplit` slices of `kslice_blocks`
   // stages (a multiple of kchunk_blocks); unit u = slice * tiles + tile writes its hi*hi sums to
   // Phh + slice * pstride and, termwise, its raw correction sums to Px + slice * pstride (both
-  // M x ldp); a reduction kernel forms C.  ksplit == 1: the kernel writes C itself.
+  // M x ldp); a reduction kernel forms C.  Phh == nullptr (then ksplit == 1): the kernel writes
+  // C itself.  Phh != nullptr with ksplit == 1 is the four-term path, whose reduction kernel
+  // adds the low-low product.
   int ksplit;
   int kslice_blocks;
   float* Phh;
@@ -476,7 +478,7 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA0, const __grid_constant__
             store16(base, ld, p.M, p.N, row, col_base + g * 16, &S[g * 16], false, accumulate);
         }
       };
-      const bool split_out = (NTERMS == 3) && (ksplit > 1);
+      const bool split_out = (NTERMS == 3) && !FUSED && (p.Phh != nullptr);
       if (split_out) store_tile(p.Phh + (long long)slice * p.pstride, p.ldp, true, 0);
       if (NTERMS == 3 && p.order == 0) {
         // Termwise: the correction stream meets the dominant stream once: here, or (split-K) in

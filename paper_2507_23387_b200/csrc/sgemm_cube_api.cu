@@ -193,7 +193,10 @@ template <int NTERMS>
 int launch_tc_gemm(sgemm_cube_ctx* h, int M, int N, int K, const uint16_t* Ahi, const uint16_t* Alo,
                    int64_t lda16, const uint16_t* Bhi, const uint16_t* Blo, int64_t ldb16, float* D,
                    int64_t ldd, int accumulate, int order, int kblock, float inv_scale,
-                   cudaStream_t st) {
+                   cudaStream_t st, const float* Dll = nullptr, int64_t ldll = 0) {
+  // Dll (NTERMS == 3, termwise only): a finished low-low product lo_A lo_B.  The kernel then
+  // writes its raw sums to the partial-sum workspace even with a single k slice and the reduction
+  // kernel forms the four-term result.
   using Cfg = sgc::TcCfg<NTERMS, false>;      // BK and the A swizzle do not depend on PAIR
   int rc = set_kernel_attrs(h);
   if (rc) return rc;
@@ -230,7 +233,7 @@ int launch_tc_gemm(sgemm_cube_ctx* h, int M, int N, int K, const uint16_t* Ahi, 
   // Split-K: when the tiles would leave more than half of the SMs idle and k is long, cut the k
   // range into slices (whole k-blocks) so that tiles x slices fills the machine; a reduction
   // kernel adds the slices' sums.
-  const bool pair = use_pair(h, M, N);
+  const bool pair = use_pair(h, M, N) && !Dll;
   if (NTERMS == 3 && h->split_k && !pair) {
     const int tiles = ((M + sgc::kBM - 1) / sgc::kBM) * ((N + sgc::kBN - 1) / sgc::kBN);
     const int num_kb = (K + Cfg::BK - 1) / Cfg::BK;
@@ -254,7 +257,16 @@ int launch_tc_gemm(sgemm_cube_ctx* h, int M, int N, int K, const uint16_t* Ahi, 
       }
     }
   }
-  if (p.ksplit > 1) {
+  if (Dll && !p.Phh) {
+    const size_t ldp = round_up((size_t)N, 4);
+    const size_t pstride = round_up((size_t)M * ldp, 64);
+    if ((rc = grow(&h->part_ws, &h->part_ws_bytes, 2 * pstride * 4))) return rc;
+    p.Phh = static_cast<float*>(h->part_ws);
+    p.Px = p.Phh + pstride;
+    p.pstride = (long long)pstride;
+    p.ldp = (long long)ldp;
+  }
+  if (p.Phh) {
     rc = launch_tc_kernel<NTERMS, false, false>(h, M, N, tmA0, tmA1, tmB0, tmB1, p, st);
     if (rc) return rc;
     const long long total = (long long)M * N;
@@ -263,7 +275,8 @@ int launch_tc_gemm(sgemm_cube_ctx* h, int M, int N, int K, const uint16_t* Ahi, 
     if (blocks > cap) blocks = cap;
     sgc::splitk_reduce_kernel<<<(unsigned)blocks, 256, 0, st>>>(M, N, p.ksplit, p.Phh, p.Px, p.pstride, p.ldp,
                                                                  D, ldd, inv_scale,
-                                                                 order == SGEMM_CUBE_TERMWISE ? 1 : 0);
+                                                                 order == SGEMM_CUBE_TERMWISE ? 1 : 0, Dll,
+                                                                 (long long)ldll);
     h->launches++;
     return cudaGetLastError() == cudaSuccess ? SGEMM_CUBE_OK : SGEMM_CUBE_CUDA_ERROR;
   }
@@ -559,6 +572,38 @@ int sgemm_cube_unfused(sgemm_cube_handle h, int M, int N, int K, const float* A,
   sgc::combine_kernel<<<(unsigned)blocks, 256, 0, st>>>(M, N, Dhh, Dx, (long long)ldD, C, ldc, inv);
   h->launches++;
   return cudaGetLastError() == cudaSuccess ? SGEMM_CUBE_OK : SGEMM_CUBE_CUDA_ERROR;
+}
+
+int sgemm_cube_four_term(sgemm_cube_handle h, int M, int N, int K, const float* A, int64_t lda,
+                         const float* B, int64_t ldb, float* C, int64_t ldc, int scale_exp,
+                         void* stream) {
+  if (!h || !A || !B || !C) return SGEMM_CUBE_INVALID_ARG;
+  int rc = check_gemm_dims(M, N, K, lda, ldb, ldc);
+  if (rc) return rc;
+  if (scale_exp < 0 || scale_exp > 24) return SGEMM_CUBE_INVALID_ARG;
+  DeviceGuard g(h->device);
+  if (!g.ok) return SGEMM_CUBE_CUDA_ERROR;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  // Workspace layout: A_hi, A_lo (M x ldA16), B_hi, B_lo (K x ldB16), D_ll (M x ldD).
+  const size_t ldA16 = round_up((size_t)K, 8), ldB16 = round_up((size_t)N, 8);
+  const size_t ldD = round_up((size_t)N, 4);
+  const size_t szA = round_up((size_t)M * ldA16 * 2, 256), szB = round_up((size_t)K * ldB16 * 2, 256);
+  const size_t szD = round_up((size_t)M * ldD * 4, 256);
+  rc = grow(&h->ws, &h->ws_bytes, 2 * szA + 2 * szB + szD);
+  if (rc) return rc;
+  uint8_t* w = static_cast<uint8_t*>(h->ws);
+  uint16_t* Ahi = reinterpret_cast<uint16_t*>(w);
+  uint16_t* Alo = reinterpret_cast<uint16_t*>(w + szA);
+  uint16_t* Bhi = reinterpret_cast<uint16_t*>(w + 2 * szA);
+  uint16_t* Blo = reinterpret_cast<uint16_t*>(w + 2 * szA + szB);
+  float* Dll = reinterpret_cast<float*>(w + 2 * szA + 2 * szB);
+  const int kb = h->kblock_termwise;
+  if ((rc = launch_split(h, M, K, A, lda, Ahi, Alo, (int64_t)ldA16, scale_exp, st))) return rc;
+  if ((rc = launch_split(h, K, N, B, ldb, Bhi, Blo, (int64_t)ldB16, scale_exp, st))) return rc;
+  if ((rc = launch_tc_gemm<1>(h, M, N, K, Alo, nullptr, ldA16, Blo, nullptr, ldB16, Dll, ldD, 0, 0, kb, 1.f, st)))
+    return rc;
+  return launch_tc_gemm<3>(h, M, N, K, Ahi, Alo, (int64_t)ldA16, Bhi, Blo, (int64_t)ldB16, C, ldc, 0,
+                           SGEMM_CUBE_TERMWISE, kb, ldexpf(1.0f, -scale_exp), st, Dll, (int64_t)ldD);
 }
 
 int sgemm_cube_host(sgemm_cube_handle h, int M, int N, int K, const float* A_host, int64_t lda,

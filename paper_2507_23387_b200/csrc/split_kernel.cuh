@@ -135,10 +135,14 @@ exponent_window_kernel(int rows, int cols, const float* __restrict__ X, long lon
 // Split-K reduction: C = sum_s Phh[s] + inv_scale * sum_s Px[s] (termwise: the slices' hi*hi sums
 // and correction sums are added among themselves, in slice order, and meet once), or
 // C = sum_s Phh[s] (elementwise: each slice's running accumulator).  FP32 RN additions.
+// Four-term variant (Dll != nullptr, termwise): the low-low product (Eq. ll_bound's term, kept)
+// joins the corrections before they meet the dominant sum:
+//   C = sum_s Phh[s] + (inv_scale * sum_s Px[s] + inv_scale^2 * Dll).
 __global__ void __launch_bounds__(256)
 splitk_reduce_kernel(int rows, int cols, int slices, const float* __restrict__ Phh,
                      const float* __restrict__ Px, long long pstride, long long ldp,
-                     float* __restrict__ C, long long ldc, float inv_scale, int termwise) {
+                     float* __restrict__ C, long long ldc, float inv_scale, int termwise,
+                     const float* __restrict__ Dll, long long ldll) {
   const long long total = (long long)rows * cols;
   const long long stride = (long long)gridDim.x * blockDim.x;
   for (long long it = (long long)blockIdx.x * blockDim.x + threadIdx.x; it < total; it += stride) {
@@ -150,7 +154,9 @@ splitk_reduce_kernel(int rows, int cols, int slices, const float* __restrict__ P
     if (termwise) {
       float x = Px[off];
       for (int s = 1; s < slices; ++s) x = __fadd_rn(x, Px[off + s * pstride]);
-      hh = __fadd_rn(hh, __fmul_rn(x, inv_scale));
+      float small = __fmul_rn(x, inv_scale);
+      if (Dll) small = __fadd_rn(small, __fmul_rn(Dll[r * ldll + c], __fmul_rn(inv_scale, inv_scale)));
+      hh = __fadd_rn(hh, small);
     }
     C[r * ldc + c] = hh;
   }

@@ -65,3 +65,13 @@ def test_harness_errors_agree_with_the_oracle_reference(handle):
     assert abs(got["termwise_s12"] / want - 1) < 1e-3
     want_f32 = oracle.frobenius_rel_err(oracle.sgemm_f32(A, B), C64)
     assert 0.2 < got["fp32_gemm"] / want_f32 < 5
+
+
+def test_dropped_term_sweep(handle):
+    # The low-low product has leading coefficient 2^-22 (Eq. ll_bound): keeping it helps only
+    # while the FP32 accumulation error (which grows with k) is smaller than that.
+    rows = {r["k"]: r for r in accuracy_study.dropped_term_sweep(handle, ks=(8, 2048), mn=512, seeds=2)}
+    assert rows[8]["four_term_frob"] < 0.95 * rows[8]["three_term_frob"]
+    assert 0.8 < rows[2048]["four_term_frob"] / rows[2048]["three_term_frob"] < 1.05
+    for r in rows.values():
+        assert r["four_term_cw"] <= 2 * r["k"] * 2.0 ** -24 and r["three_term_cw"] <= 2 * r["k"] * 2.0 ** -24

@@ -202,3 +202,52 @@ def exponent_window(X):
 def scale_exp_bounds(e_min, e_max):
     """Eq. sf_bounds: -3 - e_min <= s_b <= 26 - e_max."""
     return -3 - e_min, 26 - e_max
+
+
+# ------------------------------------------------------------------ whole-input scaling
+# Sec. 4.2 notes that once the high word is subnormal (|x| < 2^-14) scaling the residual alone no
+# longer keeps 22 bits and that whole-input scaling is then needed, and leaves it open; Sec. 7
+# lists explicit exponent management as future work.  What follows is the plain definition of
+# that extension: operands are multiplied by powers of two (exact) before the split and the
+# product is scaled back (exact unless the FP32 result leaves the normal range).
+
+def hi_exponent_range(X):
+    """[e_min, e_max, #non-finite] over the non-zero finite entries of X, where the exponent of
+    an entry is that of its value rounded (RN-even) to an 11-bit significand, i.e. the unbiased
+    exponent its FP16 high word would have if FP16 had unbounded exponent range.  (127, -127)
+    if no entry qualifies."""
+    X = np.asarray(X, dtype=np.float32)
+    finite = np.isfinite(X)
+    x = np.abs(X[finite & (X != 0)].astype(np.float64))
+    n_bad = int((~finite).sum())
+    if x.size == 0:
+        return [127, -127, n_bad]
+    m, e = np.frexp(x)                         # x = m 2^e, m in [0.5, 1)
+    r = np.rint(m * 2048.0)                    # 11-bit significand, ties to even
+    e_hi = e - 1 + (r == 2048.0)
+    return [int(e_hi.min()), int(e_hi.max()), n_bad]
+
+
+def input_scale_exps(range_a, range_b):
+    """(p_A, p_B, s_b, protected): each operand is scaled by 2^p with p = 15 - e_max, which puts
+    its largest high word in the top normal FP16 binade; the window can then span the whole
+    normal range, for which Eq. sf_bounds leaves s_b = 11.  protected: every non-zero entry of
+    both scaled operands has a normal high word (e_min + p >= -14) and no entry is inf/NaN."""
+    ps, ok = [], True
+    for e_min, e_max, n_bad in (range_a, range_b):
+        if e_max < e_min:                      # operand has no non-zero finite entry
+            ps.append(0)
+        else:
+            p = max(-126, min(126, 15 - e_max))
+            ps.append(p)
+            ok = ok and (e_min + p >= -14) and (e_max + p <= 15)
+        ok = ok and n_bad == 0
+    return ps[0], ps[1], 11, bool(ok)
+
+
+def sgemm_cube_scaled(A, B, p_a, p_b, s=11, order=TERMWISE, kb=64):
+    """2^-(p_a + p_b) * sgemm_cube(2^p_a A, 2^p_b B): whole-input scaling around Eq. recover_eqn."""
+    A2 = np.ldexp(np.asarray(A, dtype=np.float32), int(p_a)).astype(np.float32)
+    B2 = np.ldexp(np.asarray(B, dtype=np.float32), int(p_b)).astype(np.float32)
+    C = sgemm_cube(A2, B2, s=s, order=order, kb=kb)
+    return np.ldexp(C, -(int(p_a) + int(p_b))).astype(np.float32)

@@ -41,3 +41,77 @@ def test_exponent_window_counts():
     assert oracle.exponent_window(np.zeros((2, 2), dtype=np.float32)) == [127, -127, 0, 0, 4]
     # rounding carry: 2047.9 rounds up to 2048 = 2^11
     assert oracle.exponent_window([[2047.9]])[:2] == [11, 11]
+
+
+# ------------------------------------------------------------------ whole-input scaling
+from paper_2507_23387_b200 import inputs  # noqa: E402
+
+
+def test_hi_exponent_range_agrees_with_the_fp16_window_inside_the_normal_range():
+    # Where every high word is a normal FP16 number the two notions coincide; exponent_window
+    # reads the exponent field of the (separately pinned) FP16 conversion.
+    X = inputs.exponent_spread(7, (64, 48))                      # exponents -10 .. 10
+    win = oracle.exponent_window(X)
+    assert win[2:] == [0, 0, 0]
+    assert oracle.hi_exponent_range(X) == [win[0], win[1], 0]
+
+
+def test_hi_exponent_range_rounding_cases():
+    r = oracle.hi_exponent_range
+    assert r([[1.0]]) == [0, 0, 0]
+    assert r([[np.float32(2 - 2.0 ** -11)]])[:2] == [1, 1]       # tie, rounds to even = 2.0
+    tie = np.array([[2 - 2.0 ** -11]], dtype=np.float32)
+    assert oracle.split(tie, 0)[0][0, 0] == 0x4000               # the FP16 conversion says the same
+    assert r([[np.float32(2 - 2.0 ** -10)]])[:2] == [0, 0]       # representable, stays below 2
+    assert r([[65519.0]])[:2] == [15, 15] and r([[65520.0]])[:2] == [16, 16]
+    assert r([[2.0 ** -30, -3.0, 0.0]]) == [-30, 1, 0]
+    assert r([[2.0 ** -140]])[:2] == [-140, -140]                # FP32 subnormal input
+    assert r([[0.0, np.inf, np.nan]]) == [127, -127, 2]
+
+
+def test_input_scale_exps_rule():
+    # largest high word to the top normal binade; whole normal window -> s_b = 11 (Eq. sf_bounds)
+    assert oracle.input_scale_exps([-14, 15, 0], [-14, 15, 0]) == (0, 0, 11, True)
+    assert oracle.input_scale_exps([-40, -20, 0], [3, 20, 0]) == (35, -5, 11, True)
+    assert oracle.input_scale_exps([-40, -10, 0], [0, 0, 0])[3] is False     # 31 binades: too wide
+    assert oracle.input_scale_exps([0, 0, 1], [0, 0, 0])[3] is False         # inf / NaN present
+    assert oracle.input_scale_exps([127, -127, 0], [0, 0, 0])[:2] == (0, 15)  # all-zero operand
+    lo, hi = oracle.scale_exp_bounds(-14, 15)
+    assert lo <= 11 <= hi
+
+
+def test_scaled_product_is_the_plain_one_when_no_scaling_is_asked():
+    A, B = inputs.make_pair("uniform_pm1", 3, 20, 30, 70)
+    for order in (oracle.TERMWISE, oracle.ELEMENTWISE):
+        assert np.array_equal(oracle.sgemm_cube_scaled(A, B, 0, 0, 11, order, 64),
+                              oracle.sgemm_cube(A, B, 11, order, 64))
+
+
+def test_auto_scaled_product_is_scale_covariant_bit_for_bit():
+    # Multiplying an operand by a power of two shifts its p by the same amount: the split sees
+    # identical words and the result is the same up to the (exact) power of two.
+    A, B = inputs.make_pair("normal", 4, 24, 16, 100)
+    base = None
+    for a, b in ((0, 0), (-37, 9), (20, -50), (-60, -60)):
+        A2, B2 = np.ldexp(A, a).astype(np.float32), np.ldexp(B, b).astype(np.float32)
+        pa, pb, s, _ = oracle.input_scale_exps(oracle.hi_exponent_range(A2), oracle.hi_exponent_range(B2))
+        C = oracle.sgemm_cube_scaled(A2, B2, pa, pb, s, oracle.TERMWISE, 64)
+        C0 = np.ldexp(C.astype(np.float64), -(a + b))
+        if base is None:
+            base = C0
+        assert np.array_equal(C0, base)
+
+
+def test_scaling_restores_the_accuracy_of_tiny_inputs():
+    # Entries around 2^-30: every high word is zero or subnormal, the plain method loses all
+    # accuracy (Sec. 4.2, remark after Rule 1); with whole-input scaling the error is back at the
+    # level of well-scaled inputs.
+    A = inputs.uniform_range(5, (48, 200), -30, False, stream=0)
+    B = inputs.uniform_range(5, (200, 40), -30, False, stream=1)
+    C64 = oracle.dgemm_ref(A, B, with_abs=False)
+    plain = oracle.frobenius_rel_err(oracle.sgemm_cube(A, B, 12, oracle.TERMWISE, 64), C64)
+    ra, rb = oracle.hi_exponent_range(A), oracle.hi_exponent_range(B)
+    pa, pb, s, _ = oracle.input_scale_exps(ra, rb)
+    assert pa == 15 - ra[1] and pa >= 44
+    scaled = oracle.frobenius_rel_err(oracle.sgemm_cube_scaled(A, B, pa, pb, s, oracle.TERMWISE, 64), C64)
+    assert plain > 0.5 and scaled < 5e-7

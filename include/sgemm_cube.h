@@ -252,6 +252,58 @@ int sgemm_cube_exponent_window(sgemm_cube_handle h, int rows, int cols,
 int sgemm_cube_choose_scale_exp(const int64_t* window_a, const int64_t* window_b,
                                 int* scale_exp_out, int* protected_out);
 
+/* ---- Whole-input scaling (explicit exponent management).
+ * The paper notes (Sec. 4.2, after Rule 1) that once a high word is subnormal, |x| < 2^-14,
+ * scaling the residual alone cannot keep 22 bits and that the whole input must be scaled, and
+ * leaves that outside its scope (Sec. 7 lists it as future work).  These entry points are that
+ * extension: operands are multiplied by powers of two before the split (exact) and the product
+ * is multiplied by the inverse power afterwards (exact unless the FP32 result leaves the normal
+ * range, then rounded once). */
+
+/* Range of the exponents the FP16 high words of X would have if FP16 had unbounded exponent
+ * range: the unbiased exponent of |x| rounded (RN-even) to an 11-bit significand, over the
+ * non-zero finite entries.  One pass over X; the call synchronises `stream` and writes HOST memory:
+ *   range_out[0] = e_min, range_out[1] = e_max (127 / -127 if no entry qualifies),
+ *   range_out[2] = number of inf / NaN entries.
+ *   X_dev rows x cols FP32, ldx >= cols (device, read); range_out 3 x int64 (host, written).
+ * Errors: INVALID_ARG, CUDA_ERROR. */
+int sgemm_cube_hi_exponent_range(sgemm_cube_handle h, int rows, int cols,
+                                 const float* X_dev, int64_t ldx,
+                                 int64_t* range_out, void* stream);
+
+/* Scaling exponents for a pair of operands from their ranges (host arithmetic only):
+ * p = 15 - e_max per operand (its largest high word lands in the top normal FP16 binade, nothing
+ * overflows), clamped to [-126, 126]; an operand without non-zero finite entries gets p = 0.  The
+ * scaled windows may then span the whole normal range, for which Eq. sf_bounds leaves
+ * *scale_exp_out = 11.  *protected_out (optional) = 1 if every non-zero entry of both scaled
+ * operands has a normal high word (e_min + p >= -14), i.e. each operand spans at most 30 binades,
+ * and there is no inf / NaN; else 0 (the smallest entries then keep fewer than 22 bits).
+ * Errors: INVALID_ARG. */
+int sgemm_cube_choose_input_scaling(const int64_t* range_a, const int64_t* range_b,
+                                    int* p_a_out, int* p_b_out, int* scale_exp_out,
+                                    int* protected_out);
+
+/* C = 2^-(p_a + p_b) * sgemm_cube(2^p_a A, 2^p_b B): the split kernels scale while they read, one
+ * three-product kernel, one pass over C for the way back (skipped when p_a + p_b == 0).  Always
+ * the two-phase route (FP16 words in the handle's workspace), so inputs need no alignment.
+ * p_a, p_b in [-126, 126]; the other arguments and layouts as sgemm_cube.
+ * Errors: INVALID_ARG, ALLOC_FAILED, CUDA_ERROR. */
+int sgemm_cube_scaled(sgemm_cube_handle h, int M, int N, int K,
+                      const float* A_dev, int64_t lda,
+                      const float* B_dev, int64_t ldb,
+                      float* C_dev, int64_t ldc,
+                      int p_a, int p_b, int scale_exp, int accumulation_order, void* stream);
+
+/* sgemm_cube_hi_exponent_range on A and B, sgemm_cube_choose_input_scaling, sgemm_cube_scaled in
+ * one call.  Synchronises `stream` twice (the ranges are read on the host) before it enqueues the
+ * product.  chosen_out (optional, host, 4 x int): p_a, p_b, scale exponent, protected flag.
+ * Errors: as the three calls. */
+int sgemm_cube_auto_scaled(sgemm_cube_handle h, int M, int N, int K,
+                           const float* A_dev, int64_t lda,
+                           const float* B_dev, int64_t ldb,
+                           float* C_dev, int64_t ldc,
+                           int accumulation_order, void* stream, int* chosen_out);
+
 /* Size in bytes of the fixed device scratch area used by sgemm_cube_unfused_static. */
 #define SGEMM_CUBE_STATIC_SCRATCH_BYTES (32u << 20)
 

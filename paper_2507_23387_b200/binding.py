@@ -20,7 +20,8 @@ STRATEGY_AUTO, STRATEGY_FUSED, STRATEGY_TWO_PHASE = 0, 1, 2
 
 EXPORTS = ["sgemm_cube_create", "sgemm_cube_destroy", "sgemm_cube_set_option", "sgemm_cube_split",
            "sgemm_cube", "sgemm_cube_unfused", "sgemm_cube_presplit", "sgemm_cube_hgemm",
-           "sgemm_cube_four_term",
+           "sgemm_cube_four_term", "sgemm_cube_hi_exponent_range", "sgemm_cube_choose_input_scaling",
+           "sgemm_cube_scaled", "sgemm_cube_auto_scaled",
            "sgemm_cube_host", "sgemm_cube_unfused_static", "sgemm_cube_check", "sgemm_cube_launch_count", "sgemm_cube_last_kernel_ms",
            "sgemm_cube_exponent_window", "sgemm_cube_choose_scale_exp",
            "sgemm_cube_status_string", "sgemm_cube_version"]
@@ -57,6 +58,11 @@ def load():
     lib.sgemm_cube_hgemm.argtypes = [vp, i32, i32, i32, vp, i64, vp, i64, vp, i64, i32, vp]
     lib.sgemm_cube_unfused_static.argtypes = [i32, i32, i32, vp, i64, vp, i64, vp, i64, i32, vp]
     lib.sgemm_cube_four_term.argtypes = [vp, i32, i32, i32, vp, i64, vp, i64, vp, i64, i32, vp]
+    lib.sgemm_cube_hi_exponent_range.argtypes = [vp, i32, i32, vp, i64, ctypes.POINTER(i64), vp]
+    pi = ctypes.POINTER(i32)
+    lib.sgemm_cube_choose_input_scaling.argtypes = [ctypes.POINTER(i64), ctypes.POINTER(i64), pi, pi, pi, pi]
+    lib.sgemm_cube_scaled.argtypes = [vp, i32, i32, i32, vp, i64, vp, i64, vp, i64, i32, i32, i32, i32, vp]
+    lib.sgemm_cube_auto_scaled.argtypes = [vp, i32, i32, i32, vp, i64, vp, i64, vp, i64, i32, vp, pi]
     lib.sgemm_cube_check.argtypes = [vp, vp, ctypes.POINTER(ctypes.c_uint32)]
     lib.sgemm_cube_last_kernel_ms.argtypes = [vp, ctypes.POINTER(ctypes.c_float)]
     lib.sgemm_cube_exponent_window.argtypes = [vp, i32, i32, vp, i64, ctypes.POINTER(i64), vp]
@@ -115,6 +121,17 @@ def sgemm_cube_unfused_static(A, B, C, scale_exp=11, stream=None):
                                             _dev(B, torch.float32), _ld(B), _dev(C, torch.float32),
                                             _ld(C), scale_exp, _stream_ptr(stream)),
            "sgemm_cube_unfused_static")
+
+
+def sgemm_cube_choose_input_scaling(range_a, range_b):
+    """(p_a, p_b, scale_exp, protected) for two ranges (see Handle.sgemm_cube_hi_exponent_range)."""
+    ra = (ctypes.c_int64 * 3)(*[int(v) for v in range_a])
+    rb = (ctypes.c_int64 * 3)(*[int(v) for v in range_b])
+    pa, pb, s, prot = ctypes.c_int(0), ctypes.c_int(0), ctypes.c_int(0), ctypes.c_int(0)
+    _check(load().sgemm_cube_choose_input_scaling(ra, rb, ctypes.byref(pa), ctypes.byref(pb),
+                                                  ctypes.byref(s), ctypes.byref(prot)),
+           "sgemm_cube_choose_input_scaling")
+    return int(pa.value), int(pb.value), int(s.value), bool(prot.value)
 
 
 def sgemm_cube_choose_scale_exp(window_a, window_b):
@@ -181,6 +198,36 @@ class Handle:
                                            _dev(B, torch.float32), _ld(B), _dev(C, torch.float32),
                                            _ld(C), scale_exp, _stream_ptr(stream)),
                "sgemm_cube_four_term")
+
+    def sgemm_cube_hi_exponent_range(self, X, stream=None):
+        """[e_min, e_max, #inf/NaN] of the unbounded-range high-word exponents of X."""
+        rows, cols = X.shape
+        out = (ctypes.c_int64 * 3)()
+        _check(load().sgemm_cube_hi_exponent_range(self._h, rows, cols, _dev(X, torch.float32), _ld(X),
+                                                   out, _stream_ptr(stream)),
+               "sgemm_cube_hi_exponent_range")
+        return [int(v) for v in out]
+
+    def sgemm_cube_scaled(self, A, B, C, p_a, p_b, scale_exp=11, order=TERMWISE, stream=None):
+        M, K = A.shape
+        K2, N = B.shape
+        assert K == K2 and C.shape == (M, N)
+        _check(load().sgemm_cube_scaled(self._h, M, N, K, _dev(A, torch.float32), _ld(A),
+                                        _dev(B, torch.float32), _ld(B), _dev(C, torch.float32), _ld(C),
+                                        int(p_a), int(p_b), scale_exp, order, _stream_ptr(stream)),
+               "sgemm_cube_scaled")
+
+    def sgemm_cube_auto_scaled(self, A, B, C, order=TERMWISE, stream=None):
+        """Returns (p_a, p_b, scale_exp, protected) as chosen from the operands' ranges."""
+        M, K = A.shape
+        K2, N = B.shape
+        assert K == K2 and C.shape == (M, N)
+        chosen = (ctypes.c_int * 4)()
+        _check(load().sgemm_cube_auto_scaled(self._h, M, N, K, _dev(A, torch.float32), _ld(A),
+                                             _dev(B, torch.float32), _ld(B), _dev(C, torch.float32),
+                                             _ld(C), order, _stream_ptr(stream), chosen),
+               "sgemm_cube_auto_scaled")
+        return int(chosen[0]), int(chosen[1]), int(chosen[2]), bool(chosen[3])
 
     def sgemm_cube_presplit(self, Ahi, Alo, Bhi, Blo, C, scale_exp=11, order=TERMWISE, stream=None):
         M, K = Ahi.shape

@@ -172,7 +172,7 @@ int check_gemm_dims(int M, int N, int K, int64_t lda, int64_t ldb, int64_t ldc) 
 }
 
 int launch_split(sgemm_cube_ctx* h, int rows, int cols, const float* X, int64_t ldx, uint16_t* hi,
-                 uint16_t* lo, int64_t ldh, int s, cudaStream_t st) {
+                 uint16_t* lo, int64_t ldh, int s, cudaStream_t st, float pre = 1.0f) {
   const bool vec = (cols % 8 == 0) && aligned16(X) && (ldx % 4 == 0) && aligned16(hi) &&
                    aligned16(lo) && (ldh % 8 == 0);
   const long long items = vec ? (long long)rows * (cols / 8) : (long long)rows * cols;
@@ -181,9 +181,9 @@ int launch_split(sgemm_cube_ctx* h, int rows, int cols, const float* X, int64_t 
   if (blocks > cap) blocks = cap;
   if (blocks < 1) blocks = 1;
   if (vec)
-    sgc::split_vec8_kernel<<<(unsigned)blocks, 256, 0, st>>>(rows, cols, X, ldx, hi, lo, ldh, s);
+    sgc::split_vec8_kernel<<<(unsigned)blocks, 256, 0, st>>>(rows, cols, X, ldx, hi, lo, ldh, s, pre);
   else
-    sgc::split_scalar_kernel<<<(unsigned)blocks, 256, 0, st>>>(rows, cols, X, ldx, hi, lo, ldh, s);
+    sgc::split_scalar_kernel<<<(unsigned)blocks, 256, 0, st>>>(rows, cols, X, ldx, hi, lo, ldh, s, pre);
   h->launches++;
   return cudaGetLastError() == cudaSuccess ? SGEMM_CUBE_OK : SGEMM_CUBE_CUDA_ERROR;
 }
@@ -312,7 +312,8 @@ int launch_fused(sgemm_cube_ctx* h, int M, int N, int K, const float* A, int64_t
 // sgemm_cube, strategy "two-phase": split both operands once into the handle's workspace, then one
 // three-product kernel on the FP16 words.  Same arithmetic and bracketing as the fused kernel.
 int launch_two_phase(sgemm_cube_ctx* h, int M, int N, int K, const float* A, int64_t lda, const float* B,
-                     int64_t ldb, float* C, int64_t ldc, int s, int order, cudaStream_t st) {
+                     int64_t ldb, float* C, int64_t ldc, int s, int order, cudaStream_t st,
+                     float pre_a = 1.0f, float pre_b = 1.0f) {
   const size_t ldA16 = round_up((size_t)K, 8), ldB16 = round_up((size_t)N, 8);
   const size_t szA = round_up((size_t)M * ldA16 * 2, 256), szB = round_up((size_t)K * ldB16 * 2, 256);
   int rc = grow(&h->ws, &h->ws_bytes, 2 * szA + 2 * szB);
@@ -322,8 +323,8 @@ int launch_two_phase(sgemm_cube_ctx* h, int M, int N, int K, const float* A, int
   uint16_t* Alo = reinterpret_cast<uint16_t*>(w + szA);
   uint16_t* Bhi = reinterpret_cast<uint16_t*>(w + 2 * szA);
   uint16_t* Blo = reinterpret_cast<uint16_t*>(w + 2 * szA + szB);
-  if ((rc = launch_split(h, M, K, A, lda, Ahi, Alo, (int64_t)ldA16, s, st))) return rc;
-  if ((rc = launch_split(h, K, N, B, ldb, Bhi, Blo, (int64_t)ldB16, s, st))) return rc;
+  if ((rc = launch_split(h, M, K, A, lda, Ahi, Alo, (int64_t)ldA16, s, st, pre_a))) return rc;
+  if ((rc = launch_split(h, K, N, B, ldb, Bhi, Blo, (int64_t)ldB16, s, st, pre_b))) return rc;
   const int kblock = (order == SGEMM_CUBE_TERMWISE) ? h->kblock_termwise : h->kblock_elementwise;
   if (h->time_kernel && h->ev0) cudaEventRecord(h->ev0, st);
   rc = launch_tc_gemm<3>(h, M, N, K, Ahi, Alo, (int64_t)ldA16, Bhi, Blo, (int64_t)ldB16, C, ldc, 0, order,
@@ -776,6 +777,102 @@ int sgemm_cube_exponent_window(sgemm_cube_handle h, int rows, int cols, const fl
   }
   for (int i = 0; i < 5; ++i) window_out[i] = res[i];
   return SGEMM_CUBE_OK;
+}
+
+int sgemm_cube_hi_exponent_range(sgemm_cube_handle h, int rows, int cols, const float* X, int64_t ldx,
+                                 int64_t* range_out, void* stream) {
+  if (!h || !X || !range_out) return SGEMM_CUBE_INVALID_ARG;
+  if (rows <= 0 || cols <= 0 || ldx < cols) return SGEMM_CUBE_INVALID_ARG;
+  DeviceGuard g(h->device);
+  if (!g.ok) return SGEMM_CUBE_CUDA_ERROR;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  long long* dev = reinterpret_cast<long long*>(h->err_dev + 4);
+  const long long init[3] = {127, -127, 0};
+  if (cudaMemcpyAsync(dev, init, sizeof(init), cudaMemcpyHostToDevice, st) != cudaSuccess) {
+    cudaGetLastError();
+    return SGEMM_CUBE_CUDA_ERROR;
+  }
+  const long long total = (long long)rows * cols;
+  long long blocks = (total + 1023) / 1024;
+  const long long cap = (long long)h->sm_count * 16;
+  if (blocks > cap) blocks = cap;
+  sgc::hi_exponent_range_kernel<<<(unsigned)blocks, 256, 0, st>>>(rows, cols, X, ldx, dev);
+  h->launches++;
+  if (cudaGetLastError() != cudaSuccess) return SGEMM_CUBE_CUDA_ERROR;
+  long long res[3];
+  if (cudaMemcpyAsync(res, dev, sizeof(res), cudaMemcpyDeviceToHost, st) != cudaSuccess ||
+      cudaStreamSynchronize(st) != cudaSuccess) {
+    cudaGetLastError();
+    return SGEMM_CUBE_CUDA_ERROR;
+  }
+  for (int i = 0; i < 3; ++i) range_out[i] = res[i];
+  return SGEMM_CUBE_OK;
+}
+
+int sgemm_cube_choose_input_scaling(const int64_t* range_a, const int64_t* range_b, int* p_a_out,
+                                    int* p_b_out, int* scale_exp_out, int* protected_out) {
+  if (!range_a || !range_b || !p_a_out || !p_b_out || !scale_exp_out) return SGEMM_CUBE_INVALID_ARG;
+  bool ok = true;
+  const int64_t* rs[2] = {range_a, range_b};
+  int* ps[2] = {p_a_out, p_b_out};
+  for (int i = 0; i < 2; ++i) {
+    const int64_t e_min = rs[i][0], e_max = rs[i][1];
+    int p = 0;
+    if (e_max >= e_min) {                        // the operand has a non-zero finite entry
+      int64_t q = 15 - e_max;                    // largest high word into the top normal binade
+      if (q > 126) q = 126;
+      if (q < -126) q = -126;
+      p = (int)q;
+      ok = ok && (e_min + p >= -14) && (e_max + p <= 15);
+    }
+    ok = ok && rs[i][2] == 0;
+    *ps[i] = p;
+  }
+  *scale_exp_out = 11;                           // Eq. sf_bounds for the whole normal window
+  if (protected_out) *protected_out = ok ? 1 : 0;
+  return SGEMM_CUBE_OK;
+}
+
+int sgemm_cube_scaled(sgemm_cube_handle h, int M, int N, int K, const float* A, int64_t lda,
+                      const float* B, int64_t ldb, float* C, int64_t ldc, int p_a, int p_b,
+                      int scale_exp, int order, void* stream) {
+  if (!h || !A || !B || !C) return SGEMM_CUBE_INVALID_ARG;
+  int rc = check_gemm_dims(M, N, K, lda, ldb, ldc);
+  if (rc) return rc;
+  if (scale_exp < 0 || scale_exp > 24) return SGEMM_CUBE_INVALID_ARG;
+  if (order != SGEMM_CUBE_TERMWISE && order != SGEMM_CUBE_ELEMENTWISE) return SGEMM_CUBE_INVALID_ARG;
+  if (p_a < -126 || p_a > 126 || p_b < -126 || p_b > 126) return SGEMM_CUBE_INVALID_ARG;
+  DeviceGuard g(h->device);
+  if (!g.ok) return SGEMM_CUBE_CUDA_ERROR;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  rc = launch_two_phase(h, M, N, K, A, lda, B, ldb, C, ldc, scale_exp, order, st, ldexpf(1.0f, p_a),
+                        ldexpf(1.0f, p_b));
+  if (rc) return rc;
+  if (p_a + p_b != 0) {
+    const long long total = (long long)M * N;
+    long long blocks = (total + 255) / 256;
+    const long long cap = (long long)h->sm_count * 16;
+    if (blocks > cap) blocks = cap;
+    sgc::scale_pow2_kernel<<<(unsigned)blocks, 256, 0, st>>>(M, N, C, ldc, -(p_a + p_b));
+    h->launches++;
+    if (cudaGetLastError() != cudaSuccess) return SGEMM_CUBE_CUDA_ERROR;
+  }
+  return SGEMM_CUBE_OK;
+}
+
+int sgemm_cube_auto_scaled(sgemm_cube_handle h, int M, int N, int K, const float* A, int64_t lda,
+                           const float* B, int64_t ldb, float* C, int64_t ldc, int order, void* stream,
+                           int* chosen_out) {
+  if (!h || !A || !B || !C) return SGEMM_CUBE_INVALID_ARG;
+  int rc = check_gemm_dims(M, N, K, lda, ldb, ldc);
+  if (rc) return rc;
+  int64_t ra[3], rb[3];
+  if ((rc = sgemm_cube_hi_exponent_range(h, M, K, A, lda, ra, stream))) return rc;
+  if ((rc = sgemm_cube_hi_exponent_range(h, K, N, B, ldb, rb, stream))) return rc;
+  int p_a = 0, p_b = 0, s = 11, prot = 0;
+  if ((rc = sgemm_cube_choose_input_scaling(ra, rb, &p_a, &p_b, &s, &prot))) return rc;
+  if (chosen_out) { chosen_out[0] = p_a; chosen_out[1] = p_b; chosen_out[2] = s; chosen_out[3] = prot; }
+  return sgemm_cube_scaled(h, M, N, K, A, lda, B, ldb, C, ldc, p_a, p_b, s, order, stream);
 }
 
 int sgemm_cube_choose_scale_exp(const int64_t* window_a, const int64_t* window_b, int* scale_exp_out,

@@ -39,8 +39,9 @@ __device__ __forceinline__ float pow2f(int s) { return __int_as_float((127 + s) 
 __global__ void __launch_bounds__(256)
 split_vec8_kernel(int rows, int cols, const float* __restrict__ X, long long ldx,
                   uint16_t* __restrict__ hi, uint16_t* __restrict__ lo, long long ldh,
-                  int scale_exp) {
+                  int scale_exp, float pre) {
   const float scale = pow2f(scale_exp);
+  const bool prescale = pre != 1.0f;            // whole-input scaling: x 2^p before the split
   const long long items_per_row = cols >> 3;
   const long long total = (long long)rows * items_per_row;
   const long long stride = (long long)gridDim.x * blockDim.x;
@@ -48,8 +49,12 @@ split_vec8_kernel(int rows, int cols, const float* __restrict__ X, long long ldx
     const long long r = it / items_per_row;
     const long long c = (it - r * items_per_row) << 3;
     const float4* src = reinterpret_cast<const float4*>(X + r * ldx + c);
-    const float4 a = __ldg(src);
-    const float4 b = __ldg(src + 1);
+    float4 a = __ldg(src);
+    float4 b = __ldg(src + 1);
+    if (prescale) {
+      a.x = __fmul_rn(a.x, pre); a.y = __fmul_rn(a.y, pre); a.z = __fmul_rn(a.z, pre); a.w = __fmul_rn(a.w, pre);
+      b.x = __fmul_rn(b.x, pre); b.y = __fmul_rn(b.y, pre); b.z = __fmul_rn(b.z, pre); b.w = __fmul_rn(b.w, pre);
+    }
     uint4 h, l;
     split_two(a.x, a.y, scale, h.x, l.x);
     split_two(a.z, a.w, scale, h.y, l.y);
@@ -64,15 +69,18 @@ split_vec8_kernel(int rows, int cols, const float* __restrict__ X, long long ldx
 __global__ void __launch_bounds__(256)
 split_scalar_kernel(int rows, int cols, const float* __restrict__ X, long long ldx,
                     uint16_t* __restrict__ hi, uint16_t* __restrict__ lo, long long ldh,
-                    int scale_exp) {
+                    int scale_exp, float pre) {
   const float scale = pow2f(scale_exp);
+  const bool prescale = pre != 1.0f;
   const long long total = (long long)rows * cols;
   const long long stride = (long long)gridDim.x * blockDim.x;
   for (long long it = (long long)blockIdx.x * blockDim.x + threadIdx.x; it < total; it += stride) {
     const long long r = it / cols;
     const long long c = it - r * cols;
     uint16_t h, l;
-    split_one(X[r * ldx + c], scale, h, l);
+    float x = X[r * ldx + c];
+    if (prescale) x = __fmul_rn(x, pre);
+    split_one(x, scale, h, l);
     hi[r * ldh + c] = h;
     lo[r * ldh + c] = l;
   }
@@ -129,6 +137,62 @@ exponent_window_kernel(int rows, int cols, const float* __restrict__ X, long lon
     if (n_sub) atomicAdd(&cnt[2], (unsigned long long)n_sub);
     if (n_nonfinite) atomicAdd(&cnt[3], (unsigned long long)n_nonfinite);
     if (n_zero) atomicAdd(&cnt[4], (unsigned long long)n_zero);
+  }
+}
+
+// Range of the exponents the FP16 high words would have with unbounded exponent range: the
+// unbiased exponent of |x| rounded (RN-even) to an 11-bit significand, over the non-zero finite
+// entries.  This is what whole-input scaling (the extension Sec. 4.2 names after Rule 1) needs to
+// know: 2^p with p = 15 - e_max lifts the operand into the normal FP16 range.
+// out[0] = min, out[1] = max (initialised by the caller to +127 / -127), out[2] = number of
+// inf / NaN entries.  HBM-bound: 4 bytes read per element.
+__global__ void __launch_bounds__(256)
+hi_exponent_range_kernel(int rows, int cols, const float* __restrict__ X, long long ldx,
+                         long long* out) {
+  int emin = 127, emax = -127;
+  unsigned int n_bad = 0;
+  const long long total = (long long)rows * cols;
+  const long long stride = (long long)gridDim.x * blockDim.x;
+  for (long long it = (long long)blockIdx.x * blockDim.x + threadIdx.x; it < total; it += stride) {
+    const long long r = it / cols;
+    const long long c = it - r * cols;
+    float x = fabsf(__ldg(X + r * ldx + c));
+    unsigned int b = __float_as_uint(x);
+    if (b >= 0x7F800000u) { ++n_bad; continue; }
+    if (b == 0) continue;
+    int adj = 0;
+    if (b < 0x00800000u) {                       // FP32 subnormal: normalise first (exact)
+      b = __float_as_uint(__fmul_rn(x, 16777216.0f));
+      adj = -24;
+    }
+    // Adding half an ulp of the 11-bit significand carries into the exponent field exactly
+    // when the rounded value reaches the next binade (a tie there rounds to the even 1.0).
+    const int e = (int)((b + 0x1000u) >> 23) - 127 + adj;
+    emin = min(emin, e);
+    emax = max(emax, e);
+  }
+  for (int o = 16; o > 0; o >>= 1) {
+    emin = min(emin, __shfl_xor_sync(0xffffffffu, emin, o));
+    emax = max(emax, __shfl_xor_sync(0xffffffffu, emax, o));
+    n_bad += __shfl_xor_sync(0xffffffffu, n_bad, o);
+  }
+  if ((threadIdx.x & 31) == 0) {
+    atomicMin(&out[0], (long long)emin);
+    atomicMax(&out[1], (long long)emax);
+    if (n_bad) atomicAdd(reinterpret_cast<unsigned long long*>(out) + 2, (unsigned long long)n_bad);
+  }
+}
+
+// C *= 2^t, one rounding (only when the result leaves the normal FP32 range): the way back from
+// whole-input scaling.
+__global__ void __launch_bounds__(256)
+scale_pow2_kernel(int rows, int cols, float* __restrict__ C, long long ldc, int t) {
+  const long long total = (long long)rows * cols;
+  const long long stride = (long long)gridDim.x * blockDim.x;
+  for (long long it = (long long)blockIdx.x * blockDim.x + threadIdx.x; it < total; it += stride) {
+    const long long r = it / cols;
+    const long long c = it - r * cols;
+    C[r * ldc + c] = scalbnf(C[r * ldc + c], t);
   }
 }
 

@@ -65,3 +65,10 @@ def test_binding_fails_loudly_when_library_is_missing(monkeypatch, tmp_path):
     monkeypatch.setattr(binding, "LIB_PATH", str(tmp_path / "nope.so"))
     with pytest.raises(OSError):
         binding.load()
+
+
+def test_input_scaling_choice_is_host_arithmetic(lib):
+    import oracle
+    for ra, rb in [([-14, 15, 0], [-14, 15, 0]), ([-40, -20, 0], [3, 20, 0]), ([0, 0, 1], [0, 0, 0]),
+                   ([127, -127, 0], [5, 9, 0])]:
+        assert binding.sgemm_cube_choose_input_scaling(ra, rb) == oracle.input_scale_exps(ra, rb)

@@ -101,12 +101,13 @@ struct TcGemmParams {
 };
 
 #ifndef SGC_BK3
-#define SGC_BK3 32
+#define SGC_BK3 64
 #endif
 template <int NTERMS, bool PAIR = false, bool FUSED = false>
 struct TcCfg {
   // k per pipeline stage: 64 for one product; for three products 32 when the converter warps fill
-  // the stages, SGC_BK3 (32 or 16) when TMA does
+  // the stages, SGC_BK3 (64, 32 or 16) when TMA does: 64 gives two 96 KB stages (three 64 KB ones
+  // for CTA pairs) and measured 1-3 % faster than four stages of 32 across sizes; 16 much slower
   static constexpr int BK = (NTERMS == 1) ? 64 : (FUSED ? 32 : SGC_BK3);
   static constexpr int BN_CTA = PAIR ? kBN / 2 : kBN;     // B columns held by one CTA
   static constexpr int A_ROW_BYTES = BK * 2;              // 128 or 64: also the swizzle span of A
@@ -572,17 +573,24 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA0, const __grid_constant__
             }
             const uint32_t a_hi = st, a_lo = st + Cfg::A_TILE;
             const uint32_t b_hi = st + 2 * Cfg::A_TILE, b_lo = b_hi + Cfg::B_TILE;
+            // Order inside the correction chain: per 32 k-steps, lo*hi of both k16 steps, then
+            // hi*lo of both.  Fixed whatever the stage depth, so that every variant of the
+            // kernel rounds the chain identically.
+            constexpr int G = (BK < 32 ? BK : 32) / 16;
 #pragma unroll
-            for (int j = 0; j < BK / 16; ++j) {
-              const uint64_t da = umma_smem_desc(a_lo + j * 32, 16, a_sbo, a_swz);
-              const uint64_t db = umma_smem_desc(b_hi + j * 2048, b_lbo, b_sbo, kSwizzle128);
-              mma(d_x, da, db, (x_fresh && first_kb && j == 0) ? 0u : 1u);
-            }
+            for (int j0 = 0; j0 < BK / 16; j0 += G) {
 #pragma unroll
-            for (int j = 0; j < BK / 16; ++j) {
-              const uint64_t da = umma_smem_desc(a_hi + j * 32, 16, a_sbo, a_swz);
-              const uint64_t db = umma_smem_desc(b_lo + j * 2048, b_lbo, b_sbo, kSwizzle128);
-              mma(d_x, da, db, 1u);
+              for (int j = j0; j < j0 + G; ++j) {
+                const uint64_t da = umma_smem_desc(a_lo + j * 32, 16, a_sbo, a_swz);
+                const uint64_t db = umma_smem_desc(b_hi + j * 2048, b_lbo, b_sbo, kSwizzle128);
+                mma(d_x, da, db, (x_fresh && first_kb && j == 0) ? 0u : 1u);
+              }
+#pragma unroll
+              for (int j = j0; j < j0 + G; ++j) {
+                const uint64_t da = umma_smem_desc(a_hi + j * 32, 16, a_sbo, a_swz);
+                const uint64_t db = umma_smem_desc(b_lo + j * 2048, b_lbo, b_sbo, kSwizzle128);
+                mma(d_x, da, db, 1u);
+              }
             }
             return true;
           };
@@ -607,7 +615,8 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA0, const __grid_constant__
             return true;
           };
           int kb = kb_begin;
-          constexpr int kLook = PAIR ? 3 : 2;      // stages whose correction products go first
+          // stages whose correction products go first (96 or 64 k-steps' worth)
+          constexpr int kLook = ((PAIR ? 3 : 2) * 32 + BK - 1) / BK;
           if (NTERMS == 3 && p.order == 0 && kb + kLook <= kb_end) {
             // Start of a termwise k-block: the correction products of the first kLook stages go
             // first.  They do not touch region 0, so the accumulate warps get 8 kLook MMAs' worth

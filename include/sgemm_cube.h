@@ -90,7 +90,7 @@ enum {
    *                               had, FUSED otherwise (measured crossover: 512^3). */
   SGEMM_CUBE_OPT_STRATEGY = 3,
   /* 1: sgemm_cube records CUDA events around its tensor-core kernel, for
-   * sgemm_cube_last_kernel_ms.  Default 0. */
+   * sgemm_cube_last_kernel_ms and sgemm_cube_mean_kernel_ms.  Default 0. */
   SGEMM_CUBE_OPT_TIME_KERNEL = 4,
   /* 1 (default): when a problem has so few 128 x 256 tiles that more than half of the SMs would
    * idle and k is long enough, the three-product kernel (two-phase sgemm_cube,
@@ -351,6 +351,13 @@ int64_t sgemm_cube_launch_count(sgemm_cube_handle h);
  * (requires SGEMM_CUBE_OPT_TIME_KERNEL = 1 before that call; waits for the kernel to finish).
  * Errors: INVALID_ARG (timing off, or no call yet), CUDA_ERROR. */
 int sgemm_cube_last_kernel_ms(sgemm_cube_handle h, float* ms_out);
+
+/* Mean device time, in milliseconds, of the tensor-core kernel over the sgemm_cube calls made
+ * since SGEMM_CUBE_OPT_TIME_KERNEL was set to 1 or since the previous call of this function (at
+ * most the 128 most recent ones: one CUDA event pair is kept per call); *calls_out (optional) =
+ * how many calls were averaged.  Waits for those kernels to finish, then starts a new average.
+ * Errors: INVALID_ARG (timing off, or no call since), CUDA_ERROR. */
+int sgemm_cube_mean_kernel_ms(sgemm_cube_handle h, float* mean_ms_out, int* calls_out);
 
 /* Text for a status code (static storage; never NULL). */
 const char* sgemm_cube_status_string(int status);

@@ -22,7 +22,7 @@ EXPORTS = ["sgemm_cube_create", "sgemm_cube_destroy", "sgemm_cube_set_option", "
            "sgemm_cube", "sgemm_cube_unfused", "sgemm_cube_presplit", "sgemm_cube_hgemm",
            "sgemm_cube_four_term", "sgemm_cube_hi_exponent_range", "sgemm_cube_choose_input_scaling",
            "sgemm_cube_scaled", "sgemm_cube_auto_scaled",
-           "sgemm_cube_host", "sgemm_cube_unfused_static", "sgemm_cube_check", "sgemm_cube_launch_count", "sgemm_cube_last_kernel_ms",
+           "sgemm_cube_host", "sgemm_cube_unfused_static", "sgemm_cube_check", "sgemm_cube_launch_count", "sgemm_cube_last_kernel_ms", "sgemm_cube_mean_kernel_ms",
            "sgemm_cube_exponent_window", "sgemm_cube_choose_scale_exp",
            "sgemm_cube_status_string", "sgemm_cube_version"]
 
@@ -65,6 +65,7 @@ def load():
     lib.sgemm_cube_auto_scaled.argtypes = [vp, i32, i32, i32, vp, i64, vp, i64, vp, i64, i32, vp, pi]
     lib.sgemm_cube_check.argtypes = [vp, vp, ctypes.POINTER(ctypes.c_uint32)]
     lib.sgemm_cube_last_kernel_ms.argtypes = [vp, ctypes.POINTER(ctypes.c_float)]
+    lib.sgemm_cube_mean_kernel_ms.argtypes = [vp, ctypes.POINTER(ctypes.c_float), ctypes.POINTER(i32)]
     lib.sgemm_cube_exponent_window.argtypes = [vp, i32, i32, vp, i64, ctypes.POINTER(i64), vp]
     lib.sgemm_cube_choose_scale_exp.argtypes = [ctypes.POINTER(i64), ctypes.POINTER(i64),
                                                 ctypes.POINTER(i32), ctypes.POINTER(i32)]
@@ -278,3 +279,10 @@ class Handle:
         ms = ctypes.c_float(0.0)
         _check(load().sgemm_cube_last_kernel_ms(self._h, ctypes.byref(ms)), "sgemm_cube_last_kernel_ms")
         return float(ms.value)
+
+    def sgemm_cube_mean_kernel_ms(self):
+        """(mean ms, calls averaged) over the timed sgemm_cube calls since the last query."""
+        ms, n = ctypes.c_float(0.0), ctypes.c_int(0)
+        _check(load().sgemm_cube_mean_kernel_ms(self._h, ctypes.byref(ms), ctypes.byref(n)),
+               "sgemm_cube_mean_kernel_ms")
+        return float(ms.value), int(n.value)

@@ -55,8 +55,9 @@ struct sgemm_cube_ctx {
   int cta_pair = 0;            // 0/1: never/always 2-CTA clusters (cta_group::2); 2: by problem size
   int strategy = 0;            // sgemm_cube: 0 auto, 1 fused kernel, 2 split kernel + 3-product kernel
   int time_kernel = 0;         // record events around the tensor-core kernel of sgemm_cube
-  cudaEvent_t ev0 = nullptr, ev1 = nullptr;
-  bool ev_recorded = false;
+  static constexpr int kTimedCalls = 128;           // event pairs kept (most recent calls)
+  cudaEvent_t ev_ring[2 * kTimedCalls] = {};
+  long long ev_calls = 0;      // timed calls since timing was switched on or last averaged
   // host-buffer path: copy streams and events of the panel pipeline (created on first use)
   static constexpr int kMaxPanels = 32;
   cudaStream_t s_in = nullptr, s_out = nullptr;
@@ -326,10 +327,11 @@ int launch_two_phase(sgemm_cube_ctx* h, int M, int N, int K, const float* A, int
   if ((rc = launch_split(h, M, K, A, lda, Ahi, Alo, (int64_t)ldA16, s, st, pre_a))) return rc;
   if ((rc = launch_split(h, K, N, B, ldb, Bhi, Blo, (int64_t)ldB16, s, st, pre_b))) return rc;
   const int kblock = (order == SGEMM_CUBE_TERMWISE) ? h->kblock_termwise : h->kblock_elementwise;
-  if (h->time_kernel && h->ev0) cudaEventRecord(h->ev0, st);
+  const int slot = (int)(h->ev_calls % sgemm_cube_ctx::kTimedCalls);
+  if (h->time_kernel) cudaEventRecord(h->ev_ring[2 * slot], st);
   rc = launch_tc_gemm<3>(h, M, N, K, Ahi, Alo, (int64_t)ldA16, Bhi, Blo, (int64_t)ldB16, C, ldc, 0, order,
                          kblock, ldexpf(1.0f, -s), st);
-  if (h->time_kernel && h->ev1) { cudaEventRecord(h->ev1, st); h->ev_recorded = true; }
+  if (h->time_kernel) { cudaEventRecord(h->ev_ring[2 * slot + 1], st); h->ev_calls++; }
   return rc;
 }
 
@@ -346,9 +348,10 @@ int launch_sgemm_cube(sgemm_cube_ctx* h, int M, int N, int K, const float* A, in
     if (rc != SGEMM_CUBE_ALLOC_FAILED || h->strategy == 2) return rc;
     // no room for the FP16 words: the fused kernel needs no workspace
   }
-  if (h->time_kernel && h->ev0) cudaEventRecord(h->ev0, st);
+  const int slot = (int)(h->ev_calls % sgemm_cube_ctx::kTimedCalls);
+  if (h->time_kernel) cudaEventRecord(h->ev_ring[2 * slot], st);
   int rc = launch_fused(h, M, N, K, A, lda, B, ldb, C, ldc, s, order, st);
-  if (h->time_kernel && h->ev1) { cudaEventRecord(h->ev1, st); h->ev_recorded = true; }
+  if (h->time_kernel) { cudaEventRecord(h->ev_ring[2 * slot + 1], st); h->ev_calls++; }
   return rc;
 }
 
@@ -425,8 +428,8 @@ int sgemm_cube_destroy(sgemm_cube_handle h) {
   if (h->ws) cudaFree(h->ws);
   if (h->host_ws) cudaFree(h->host_ws);
   if (h->part_ws) cudaFree(h->part_ws);
-  if (h->ev0) cudaEventDestroy(h->ev0);
-  if (h->ev1) cudaEventDestroy(h->ev1);
+  for (cudaEvent_t e : h->ev_ring)
+    if (e) cudaEventDestroy(e);
   if (h->s_in) cudaStreamDestroy(h->s_in);
   if (h->s_out) cudaStreamDestroy(h->s_out);
   if (h->ev_start) cudaEventDestroy(h->ev_start);
@@ -461,14 +464,20 @@ int sgemm_cube_set_option(sgemm_cube_handle h, int option, int64_t value) {
   if (option == SGEMM_CUBE_OPT_TIME_KERNEL) {
     if (value != 0 && value != 1) return SGEMM_CUBE_INVALID_ARG;
     DeviceGuard g(h->device);
-    if (value && !h->ev0) {
-      if (cudaEventCreate(&h->ev0) != cudaSuccess || cudaEventCreate(&h->ev1) != cudaSuccess) {
-        cudaGetLastError();
-        return SGEMM_CUBE_CUDA_ERROR;
+    if (value && !h->ev_ring[0]) {
+      for (cudaEvent_t& e : h->ev_ring) {
+        if (cudaEventCreate(&e) != cudaSuccess) {
+          cudaGetLastError();
+          for (cudaEvent_t& d : h->ev_ring) {
+            if (d) cudaEventDestroy(d);
+            d = nullptr;
+          }
+          return SGEMM_CUBE_CUDA_ERROR;
+        }
       }
     }
     h->time_kernel = (int)value;
-    h->ev_recorded = false;
+    h->ev_calls = 0;
     return SGEMM_CUBE_OK;
   }
   if (value < 64 || value % 64 != 0 || value > (1 << 24)) return SGEMM_CUBE_INVALID_ARG;
@@ -903,13 +912,35 @@ int sgemm_cube_choose_scale_exp(const int64_t* window_a, const int64_t* window_b
 int64_t sgemm_cube_launch_count(sgemm_cube_handle h) { return h ? h->launches : -1; }
 
 int sgemm_cube_last_kernel_ms(sgemm_cube_handle h, float* ms_out) {
-  if (!h || !ms_out || !h->time_kernel || !h->ev_recorded) return SGEMM_CUBE_INVALID_ARG;
+  if (!h || !ms_out || !h->time_kernel || h->ev_calls == 0) return SGEMM_CUBE_INVALID_ARG;
   DeviceGuard g(h->device);
-  if (cudaEventSynchronize(h->ev1) != cudaSuccess ||
-      cudaEventElapsedTime(ms_out, h->ev0, h->ev1) != cudaSuccess) {
+  const int slot = (int)((h->ev_calls - 1) % sgemm_cube_ctx::kTimedCalls);
+  if (cudaEventSynchronize(h->ev_ring[2 * slot + 1]) != cudaSuccess ||
+      cudaEventElapsedTime(ms_out, h->ev_ring[2 * slot], h->ev_ring[2 * slot + 1]) != cudaSuccess) {
     cudaGetLastError();
     return SGEMM_CUBE_CUDA_ERROR;
   }
+  return SGEMM_CUBE_OK;
+}
+
+int sgemm_cube_mean_kernel_ms(sgemm_cube_handle h, float* mean_ms_out, int* calls_out) {
+  if (!h || !mean_ms_out || !h->time_kernel || h->ev_calls == 0) return SGEMM_CUBE_INVALID_ARG;
+  DeviceGuard g(h->device);
+  const long long n = h->ev_calls < sgemm_cube_ctx::kTimedCalls ? h->ev_calls : sgemm_cube_ctx::kTimedCalls;
+  double sum = 0.0;
+  for (long long i = 0; i < n; ++i) {
+    const int slot = (int)((h->ev_calls - 1 - i) % sgemm_cube_ctx::kTimedCalls);
+    float ms = 0.f;
+    if (cudaEventSynchronize(h->ev_ring[2 * slot + 1]) != cudaSuccess ||
+        cudaEventElapsedTime(&ms, h->ev_ring[2 * slot], h->ev_ring[2 * slot + 1]) != cudaSuccess) {
+      cudaGetLastError();
+      return SGEMM_CUBE_CUDA_ERROR;
+    }
+    sum += ms;
+  }
+  *mean_ms_out = (float)(sum / (double)n);
+  if (calls_out) *calls_out = (int)n;
+  h->ev_calls = 0;
   return SGEMM_CUBE_OK;
 }
 

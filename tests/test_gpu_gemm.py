@@ -365,3 +365,28 @@ def test_host_buffer_entry_point(handle, shape):
     C2 = torch.empty((M, N))
     handle.sgemm_cube_host(torch.from_numpy(A), torch.from_numpy(B), C2, 11, T)
     assert np.array_equal(C2.numpy(), run(handle, "auto", padded_dev(A, 4), padded_dev(B, 4), 11, T))
+
+
+def test_kernel_timing_queries(handle):
+    A, B = inputs.make_pair("uniform_pm1", 2, 512, 512, 512)
+    Ad, Bd = to_dev(A), to_dev(B)
+    C = torch.empty((512, 512), device="cuda:0")
+    with pytest.raises(binding.SgemmCubeError):
+        handle.sgemm_cube_last_kernel_ms()                   # timing is off by default
+    handle.sgemm_cube_set_option(binding.OPT_TIME_KERNEL, 1)
+    try:
+        with pytest.raises(binding.SgemmCubeError):
+            handle.sgemm_cube_mean_kernel_ms()               # no timed call yet
+        for _ in range(3):
+            handle.sgemm_cube(Ad, Bd, C, 11, T)
+        last = handle.sgemm_cube_last_kernel_ms()
+        mean, n = handle.sgemm_cube_mean_kernel_ms()
+        assert n == 3 and 0 < mean < 50 and 0 < last < 50
+        with pytest.raises(binding.SgemmCubeError):
+            handle.sgemm_cube_mean_kernel_ms()               # the average restarts after a query
+        for _ in range(130):                                  # more calls than event pairs are kept
+            handle.sgemm_cube(Ad, Bd, C, 11, T)
+        mean, n = handle.sgemm_cube_mean_kernel_ms()
+        assert n == 128 and 0 < mean < 50
+    finally:
+        handle.sgemm_cube_set_option(binding.OPT_TIME_KERNEL, 0)

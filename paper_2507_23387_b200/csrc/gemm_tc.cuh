@@ -537,6 +537,21 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA0, const __grid_constant__
       constexpr uint32_t a_sbo = 8 * Cfg::A_ROW_BYTES;     // 8 rows of the swizzle atom
       constexpr uint32_t b_lbo = BK * 128;                 // next 64-column atom of B
       constexpr uint32_t b_sbo = 1024;                     // next 8 k-rows inside an atom
+      // The issuing thread is a single lane: every instruction it spends on a descriptor delays
+      // the next MMA.  Only the start-address field (low word, in units of 16 bytes) changes from
+      // one MMA to the next, so the constant fields are folded at compile time and a descriptor
+      // costs one 32-bit add.
+      constexpr uint32_t a_desc_hi =
+          ((a_sbo >> 4) & 0x3FFFu) | (1u << 14) | ((uint32_t)a_swz << 29);
+      constexpr uint32_t b_desc_hi =
+          ((b_sbo >> 4) & 0x3FFFu) | (1u << 14) | ((uint32_t)kSwizzle128 << 29);
+      constexpr uint32_t a_desc_lo0 = ((16u >> 4) & 0x3FFFu) << 16;
+      constexpr uint32_t b_desc_lo0 = ((b_lbo >> 4) & 0x3FFFu) << 16;
+      auto desc = [](uint32_t lo, uint32_t hi) -> uint64_t {
+        uint64_t d;
+        asm("mov.b64 %0, {%1, %2};" : "=l"(d) : "r"(lo), "r"(hi));
+        return d;
+      };
       uint32_t it = 0;
       uint32_t fills[2] = {0, 0};     // how many times each TMEM region has been handed over
       uint32_t gchunk = 0;            // running k-block counter (NTERMS == 1 region choice)
@@ -571,8 +586,9 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA0, const __grid_constant__
               tc_fence_after_sync();
               x_ready = true;
             }
-            const uint32_t a_hi = st, a_lo = st + Cfg::A_TILE;
-            const uint32_t b_hi = st + 2 * Cfg::A_TILE, b_lo = b_hi + Cfg::B_TILE;
+            const uint32_t a_hi = a_desc_lo0 + (st >> 4), a_lo = a_hi + (Cfg::A_TILE >> 4);
+            const uint32_t b_hi = b_desc_lo0 + ((st + 2 * Cfg::A_TILE) >> 4);
+            const uint32_t b_lo = b_hi + (Cfg::B_TILE >> 4);
             // Order inside the correction chain: per 32 k-steps, lo*hi of both k16 steps, then
             // hi*lo of both.  Fixed whatever the stage depth, so that every variant of the
             // kernel rounds the chain identically.
@@ -581,14 +597,14 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA0, const __grid_constant__
             for (int j0 = 0; j0 < BK / 16; j0 += G) {
 #pragma unroll
               for (int j = j0; j < j0 + G; ++j) {
-                const uint64_t da = umma_smem_desc(a_lo + j * 32, 16, a_sbo, a_swz);
-                const uint64_t db = umma_smem_desc(b_hi + j * 2048, b_lbo, b_sbo, kSwizzle128);
+                const uint64_t da = desc(a_lo + 2 * j, a_desc_hi);
+                const uint64_t db = desc(b_hi + 128 * j, b_desc_hi);
                 mma(d_x, da, db, (x_fresh && first_kb && j == 0) ? 0u : 1u);
               }
 #pragma unroll
               for (int j = j0; j < j0 + G; ++j) {
-                const uint64_t da = umma_smem_desc(a_hi + j * 32, 16, a_sbo, a_swz);
-                const uint64_t db = umma_smem_desc(b_lo + j * 2048, b_lbo, b_sbo, kSwizzle128);
+                const uint64_t da = desc(a_hi + 2 * j, a_desc_hi);
+                const uint64_t db = desc(b_lo + 128 * j, b_desc_hi);
                 mma(d_x, da, db, 1u);
               }
             }
@@ -603,12 +619,12 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA0, const __grid_constant__
               tc_fence_after_sync();
               main_ready = true;
             }
-            const uint32_t a_hi = st;
-            const uint32_t b_hi = st + ((NTERMS == 3) ? 2 * Cfg::A_TILE : Cfg::A_TILE);
+            const uint32_t a_hi = a_desc_lo0 + (st >> 4);
+            const uint32_t b_hi = b_desc_lo0 + ((st + ((NTERMS == 3) ? 2 * Cfg::A_TILE : Cfg::A_TILE)) >> 4);
 #pragma unroll
             for (int j = 0; j < BK / 16; ++j) {
-              const uint64_t da = umma_smem_desc(a_hi + j * 32, 16, a_sbo, a_swz);
-              const uint64_t db = umma_smem_desc(b_hi + j * 2048, b_lbo, b_sbo, kSwizzle128);
+              const uint64_t da = desc(a_hi + 2 * j, a_desc_hi);
+              const uint64_t db = desc(b_hi + 128 * j, b_desc_hi);
               mma(d_main, da, db, (first_kb && j == 0) ? 0u : 1u);
             }
             commit_both(&empty_bar[i % STAGES]);   // the stage may be refilled once these MMAs retire
@@ -616,7 +632,11 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA0, const __grid_constant__
           };
           int kb = kb_begin;
           // stages whose correction products go first (96 or 64 k-steps' worth)
+#ifdef SGC_KLOOK
+          constexpr int kLook = SGC_KLOOK;
+#else
           constexpr int kLook = ((PAIR ? 3 : 2) * 32 + BK - 1) / BK;
+#endif
           if (NTERMS == 3 && p.order == 0 && kb + kLook <= kb_end) {
             // Start of a termwise k-block: the correction products of the first kLook stages go
             // first.  They do not touch region 0, so the accumulate warps get 8 kLook MMAs' worth

@@ -29,7 +29,9 @@ def padded_dev(x, mult):
 
 def gates(C_gpu, A_rows, B, s, order, kb=None, label=""):
     """The three gates every CUDA result must pass on the rows it is checked on:
-       (1) componentwise  |C - C64| <= 2 K 2^-24 (|A||B|)      (covers truncating accumulation)
+       (1) componentwise  |C - C64| <= 2 K 2^-24 (|A||B|)      (covers truncating accumulation;
+           for K < 14 the representation error outweighs the accumulation error and the bound is
+           the first-order form of Eq. main_bound, (K + 14) 2^-24, which equals 2 K 2^-24 at K = 14)
        (2) eta_gpu  <= 2 x eta_oracle,  (3) frob_gpu <= 2 x frob_oracle, the oracle run in the same
        order with the same k-block (the larger of that and the plain sequential sum, kb = K)."""
     K = A_rows.shape[1]
@@ -44,7 +46,7 @@ def gates(C_gpu, A_rows, B, s, order, kb=None, label=""):
         frobs.append(oracle.frobenius_rel_err(Co, C64))
     msg = "%s eta_gpu=%.3e frob_gpu=%.3e oracle eta=%s frob=%s" % (label, eta_g, frob_g, etas, frobs)
     assert np.isfinite(C_gpu).all(), msg
-    assert eta_g <= 2 * K * U32, msg
+    assert eta_g <= max(2 * K, K + 14) * U32, msg
     assert eta_g <= 2 * max(etas), msg
     assert frob_g <= 2 * max(frobs), msg
     return eta_g, frob_g

@@ -122,6 +122,17 @@ def test_ragged_shapes(handle, path, order, shape):
     gates(C, A, B, 11, order, label="%s %s" % (path, shape))
 
 
+@pytest.mark.parametrize("path,order", [("fused", T), ("two_phase", T), ("two_phase", E), ("unfused", T)])
+@pytest.mark.parametrize("shape", [(100003, 8, 16), (8, 100004, 24), (4, 4, 100000), (1, 4096, 1),
+                                   (70000, 1, 1)])
+def test_extreme_aspect_ratios(handle, path, order, shape):
+    # one dimension far beyond the others: tile counts, grid sizes and 64-bit offsets
+    M, N, K = shape
+    A, B = inputs.make_pair("uniform_pm1", 13, M, N, K)
+    C = run(handle, path, padded_dev(A, 4), padded_dev(B, 4), 11, order)
+    gates(C, A, B, 11, order, label="%s %s" % (path, shape))
+
+
 @pytest.mark.parametrize("path,order", [("fused", T), ("fused", E), ("presplit", T)])
 def test_output_leading_dimension_and_alignment(handle, path, order):
     M, N, K = 150, 203, 77

@@ -127,7 +127,8 @@ int sgemm_cube_set_option(sgemm_cube_handle h, int option, int64_t value);
  * out-of-range inputs follow IEEE (|x| >= 65520 -> hi = inf, lo = NaN or inf).
  *   X_dev      rows x cols FP32, row-major, leading dimension ldx >= cols          (device, read)
  *   hi_dev/lo_dev  rows x cols FP16 bit patterns, leading dimension ldh >= cols    (device, written)
- *   scale_exp  s in [0, 24]
+ *   scale_exp  s in [0, 24];  rows, cols >= 0 (nothing is done, and the pointers are not looked
+ *   at, when either is 0)
  * Any alignment is accepted; 16-byte aligned pointers with ldx % 4 == 0 and ldh % 8 == 0 take
  * the vectorised path.  Errors: INVALID_ARG, CUDA_ERROR. */
 int sgemm_cube_split(sgemm_cube_handle h, int rows, int cols,
@@ -147,7 +148,10 @@ int sgemm_cube_split(sgemm_cube_handle h, int rows, int cols,
  *   C_dev  M x N FP32, ldc >= N     (device, written)
  *   scale_exp s in [0, 24]; accumulation_order SGEMM_CUBE_TERMWISE or SGEMM_CUBE_ELEMENTWISE
  * Alignment: A_dev, B_dev 16-byte aligned and lda % 4 == 0, ldb % 4 == 0 (else MISALIGNED).
- * C_dev may have any alignment.  M, N, K >= 1, any values (ragged edges are handled).
+ * C_dev may have any alignment.  M, N, K >= 0, any values (ragged edges are handled).  Empty
+ * problems are valid in every GEMM entry point of this header: M == 0 or N == 0 does nothing,
+ * K == 0 stores C = 0 (the empty sum; left alone by sgemm_cube_hgemm with accumulate != 0); an
+ * operand without elements may be a null pointer.
  * Errors: INVALID_ARG, MISALIGNED, CUDA_ERROR (ALLOC_FAILED only with the TWO_PHASE strategy
  * forced; AUTO falls back to the fused kernel when the workspace cannot be had). */
 int sgemm_cube(sgemm_cube_handle h, int M, int N, int K,

@@ -166,10 +166,31 @@ int launch_tc_kernel(sgemm_cube_ctx* h, int M, int N, const CUtensorMap& tmA0, c
              ? SGEMM_CUBE_OK : (cudaGetLastError(), SGEMM_CUBE_CUDA_ERROR);
 }
 
+// Dimensions may be zero (an empty operand may then be a null pointer); negative ones are errors.
 int check_gemm_dims(int M, int N, int K, int64_t lda, int64_t ldb, int64_t ldc) {
-  if (M <= 0 || N <= 0 || K <= 0) return SGEMM_CUBE_INVALID_ARG;
+  if (M < 0 || N < 0 || K < 0) return SGEMM_CUBE_INVALID_ARG;
   if (lda < K || ldb < N || ldc < N) return SGEMM_CUBE_INVALID_ARG;
   return SGEMM_CUBE_OK;
+}
+bool missing_operand(int M, int N, int K, const void* A, const void* A2, const void* B, const void* B2,
+                     const void* C) {
+  return ((!A || !A2) && M > 0 && K > 0) || ((!B || !B2) && K > 0 && N > 0) || (!C && M > 0 && N > 0);
+}
+// Empty problems: nothing to do when C has no elements; an empty inner dimension leaves the empty
+// sum, C = 0 (unless the call accumulates into C).  Returns true when the call is complete.
+bool empty_problem(int M, int N, int K, float* C, int64_t ldc, cudaStream_t st, bool c_on_host,
+                   bool keep_c, int* status) {
+  if (M > 0 && N > 0 && K > 0) return false;
+  *status = SGEMM_CUBE_OK;
+  if (M == 0 || N == 0 || keep_c) return true;
+  if (c_on_host) {
+    for (int i = 0; i < M; ++i) memset(C + (size_t)i * ldc, 0, (size_t)N * sizeof(float));
+  } else if (cudaMemset2DAsync(C, (size_t)ldc * sizeof(float), 0, (size_t)N * sizeof(float), M, st) !=
+             cudaSuccess) {
+    cudaGetLastError();
+    *status = SGEMM_CUBE_CUDA_ERROR;
+  }
+  return true;
 }
 
 int launch_split(sgemm_cube_ctx* h, int rows, int cols, const float* X, int64_t ldx, uint16_t* hi,
@@ -489,9 +510,11 @@ int sgemm_cube_set_option(sgemm_cube_handle h, int option, int64_t value) {
 
 int sgemm_cube_split(sgemm_cube_handle h, int rows, int cols, const float* X, int64_t ldx,
                      uint16_t* hi, uint16_t* lo, int64_t ldh, int scale_exp, void* stream) {
-  if (!h || !X || !hi || !lo) return SGEMM_CUBE_INVALID_ARG;
-  if (rows <= 0 || cols <= 0 || ldx < cols || ldh < cols) return SGEMM_CUBE_INVALID_ARG;
+  if (!h) return SGEMM_CUBE_INVALID_ARG;
+  if (rows < 0 || cols < 0 || ldx < cols || ldh < cols) return SGEMM_CUBE_INVALID_ARG;
   if (scale_exp < 0 || scale_exp > 24) return SGEMM_CUBE_INVALID_ARG;
+  if (rows == 0 || cols == 0) return SGEMM_CUBE_OK;
+  if (!X || !hi || !lo) return SGEMM_CUBE_INVALID_ARG;
   DeviceGuard g(h->device);
   if (!g.ok) return SGEMM_CUBE_CUDA_ERROR;
   return launch_split(h, rows, cols, X, ldx, hi, lo, ldh, scale_exp, static_cast<cudaStream_t>(stream));
@@ -499,14 +522,16 @@ int sgemm_cube_split(sgemm_cube_handle h, int rows, int cols, const float* X, in
 
 int sgemm_cube(sgemm_cube_handle h, int M, int N, int K, const float* A, int64_t lda, const float* B,
                int64_t ldb, float* C, int64_t ldc, int scale_exp, int order, void* stream) {
-  if (!h || !A || !B || !C) return SGEMM_CUBE_INVALID_ARG;
+  if (!h) return SGEMM_CUBE_INVALID_ARG;
   int rc = check_gemm_dims(M, N, K, lda, ldb, ldc);
   if (rc) return rc;
+  if (missing_operand(M, N, K, A, A, B, B, C)) return SGEMM_CUBE_INVALID_ARG;
   if (scale_exp < 0 || scale_exp > 24) return SGEMM_CUBE_INVALID_ARG;
   if (order != SGEMM_CUBE_TERMWISE && order != SGEMM_CUBE_ELEMENTWISE) return SGEMM_CUBE_INVALID_ARG;
-  if (!aligned16(A) || !aligned16(B) || (lda % 4) || (ldb % 4)) return SGEMM_CUBE_MISALIGNED;
   DeviceGuard g(h->device);
   if (!g.ok) return SGEMM_CUBE_CUDA_ERROR;
+  if (empty_problem(M, N, K, C, ldc, static_cast<cudaStream_t>(stream), false, false, &rc)) return rc;
+  if (!aligned16(A) || !aligned16(B) || (lda % 4) || (ldb % 4)) return SGEMM_CUBE_MISALIGNED;
   return launch_sgemm_cube(h, M, N, K, A, lda, B, ldb, C, ldc, scale_exp, order,
                            static_cast<cudaStream_t>(stream));
 }
@@ -514,16 +539,18 @@ int sgemm_cube(sgemm_cube_handle h, int M, int N, int K, const float* A, int64_t
 int sgemm_cube_presplit(sgemm_cube_handle h, int M, int N, int K, const uint16_t* Ahi,
                         const uint16_t* Alo, int64_t lda16, const uint16_t* Bhi, const uint16_t* Blo,
                         int64_t ldb16, float* C, int64_t ldc, int scale_exp, int order, void* stream) {
-  if (!h || !Ahi || !Alo || !Bhi || !Blo || !C) return SGEMM_CUBE_INVALID_ARG;
+  if (!h) return SGEMM_CUBE_INVALID_ARG;
   int rc = check_gemm_dims(M, N, K, lda16, ldb16, ldc);
   if (rc) return rc;
+  if (missing_operand(M, N, K, Ahi, Alo, Bhi, Blo, C)) return SGEMM_CUBE_INVALID_ARG;
   if (scale_exp < 0 || scale_exp > 24) return SGEMM_CUBE_INVALID_ARG;
   if (order != SGEMM_CUBE_TERMWISE && order != SGEMM_CUBE_ELEMENTWISE) return SGEMM_CUBE_INVALID_ARG;
+  DeviceGuard g(h->device);
+  if (!g.ok) return SGEMM_CUBE_CUDA_ERROR;
+  if (empty_problem(M, N, K, C, ldc, static_cast<cudaStream_t>(stream), false, false, &rc)) return rc;
   if (!aligned16(Ahi) || !aligned16(Alo) || !aligned16(Bhi) || !aligned16(Blo) || (lda16 % 8) ||
       (ldb16 % 8))
     return SGEMM_CUBE_MISALIGNED;
-  DeviceGuard g(h->device);
-  if (!g.ok) return SGEMM_CUBE_CUDA_ERROR;
   const int kblock = (order == SGEMM_CUBE_TERMWISE) ? h->kblock_termwise : h->kblock_elementwise;
   return launch_tc_gemm<3>(h, M, N, K, Ahi, Alo, lda16, Bhi, Blo, ldb16, C, ldc, 0, order, kblock,
                            ldexpf(1.0f, -scale_exp), static_cast<cudaStream_t>(stream));
@@ -532,12 +559,14 @@ int sgemm_cube_presplit(sgemm_cube_handle h, int M, int N, int K, const uint16_t
 int sgemm_cube_hgemm(sgemm_cube_handle h, int M, int N, int K, const uint16_t* A16, int64_t lda16,
                      const uint16_t* B16, int64_t ldb16, float* D, int64_t ldd, int accumulate,
                      void* stream) {
-  if (!h || !A16 || !B16 || !D) return SGEMM_CUBE_INVALID_ARG;
+  if (!h) return SGEMM_CUBE_INVALID_ARG;
   int rc = check_gemm_dims(M, N, K, lda16, ldb16, ldd);
   if (rc) return rc;
-  if (!aligned16(A16) || !aligned16(B16) || (lda16 % 8) || (ldb16 % 8)) return SGEMM_CUBE_MISALIGNED;
+  if (missing_operand(M, N, K, A16, A16, B16, B16, D)) return SGEMM_CUBE_INVALID_ARG;
   DeviceGuard g(h->device);
   if (!g.ok) return SGEMM_CUBE_CUDA_ERROR;
+  if (empty_problem(M, N, K, D, ldd, static_cast<cudaStream_t>(stream), false, accumulate != 0, &rc)) return rc;
+  if (!aligned16(A16) || !aligned16(B16) || (lda16 % 8) || (ldb16 % 8)) return SGEMM_CUBE_MISALIGNED;
   return launch_tc_gemm<1>(h, M, N, K, A16, nullptr, lda16, B16, nullptr, ldb16, D, ldd,
                            accumulate ? 1 : 0, 0, h->kblock_termwise, 1.0f,
                            static_cast<cudaStream_t>(stream));
@@ -546,13 +575,15 @@ int sgemm_cube_hgemm(sgemm_cube_handle h, int M, int N, int K, const uint16_t* A
 int sgemm_cube_unfused(sgemm_cube_handle h, int M, int N, int K, const float* A, int64_t lda,
                        const float* B, int64_t ldb, float* C, int64_t ldc, int scale_exp, int order,
                        void* stream) {
-  if (!h || !A || !B || !C) return SGEMM_CUBE_INVALID_ARG;
+  if (!h) return SGEMM_CUBE_INVALID_ARG;
   int rc = check_gemm_dims(M, N, K, lda, ldb, ldc);
   if (rc) return rc;
+  if (missing_operand(M, N, K, A, A, B, B, C)) return SGEMM_CUBE_INVALID_ARG;
   if (scale_exp < 0 || scale_exp > 24) return SGEMM_CUBE_INVALID_ARG;
   if (order != SGEMM_CUBE_TERMWISE) return SGEMM_CUBE_INVALID_ARG;
   DeviceGuard g(h->device);
   if (!g.ok) return SGEMM_CUBE_CUDA_ERROR;
+  if (empty_problem(M, N, K, C, ldc, static_cast<cudaStream_t>(stream), false, false, &rc)) return rc;
   cudaStream_t st = static_cast<cudaStream_t>(stream);
   // Workspace layout: A_hi, A_lo (M x ldA16), B_hi, B_lo (K x ldB16), D_hh, D_x (M x ldD).
   const size_t ldA16 = round_up((size_t)K, 8), ldB16 = round_up((size_t)N, 8);
@@ -587,12 +618,14 @@ int sgemm_cube_unfused(sgemm_cube_handle h, int M, int N, int K, const float* A,
 int sgemm_cube_four_term(sgemm_cube_handle h, int M, int N, int K, const float* A, int64_t lda,
                          const float* B, int64_t ldb, float* C, int64_t ldc, int scale_exp,
                          void* stream) {
-  if (!h || !A || !B || !C) return SGEMM_CUBE_INVALID_ARG;
+  if (!h) return SGEMM_CUBE_INVALID_ARG;
   int rc = check_gemm_dims(M, N, K, lda, ldb, ldc);
   if (rc) return rc;
+  if (missing_operand(M, N, K, A, A, B, B, C)) return SGEMM_CUBE_INVALID_ARG;
   if (scale_exp < 0 || scale_exp > 24) return SGEMM_CUBE_INVALID_ARG;
   DeviceGuard g(h->device);
   if (!g.ok) return SGEMM_CUBE_CUDA_ERROR;
+  if (empty_problem(M, N, K, C, ldc, static_cast<cudaStream_t>(stream), false, false, &rc)) return rc;
   cudaStream_t st = static_cast<cudaStream_t>(stream);
   // Workspace layout: A_hi, A_lo (M x ldA16), B_hi, B_lo (K x ldB16), D_ll (M x ldD).
   const size_t ldA16 = round_up((size_t)K, 8), ldB16 = round_up((size_t)N, 8);
@@ -619,13 +652,15 @@ int sgemm_cube_four_term(sgemm_cube_handle h, int M, int N, int K, const float* 
 int sgemm_cube_host(sgemm_cube_handle h, int M, int N, int K, const float* A_host, int64_t lda,
                     const float* B_host, int64_t ldb, float* C_host, int64_t ldc, int scale_exp,
                     int order, void* stream) {
-  if (!h || !A_host || !B_host || !C_host) return SGEMM_CUBE_INVALID_ARG;
+  if (!h) return SGEMM_CUBE_INVALID_ARG;
   int rc = check_gemm_dims(M, N, K, lda, ldb, ldc);
   if (rc) return rc;
+  if (missing_operand(M, N, K, A_host, A_host, B_host, B_host, C_host)) return SGEMM_CUBE_INVALID_ARG;
   if (scale_exp < 0 || scale_exp > 24) return SGEMM_CUBE_INVALID_ARG;
   if (order != SGEMM_CUBE_TERMWISE && order != SGEMM_CUBE_ELEMENTWISE) return SGEMM_CUBE_INVALID_ARG;
   DeviceGuard g(h->device);
   if (!g.ok) return SGEMM_CUBE_CUDA_ERROR;
+  if (empty_problem(M, N, K, C_host, ldc, static_cast<cudaStream_t>(stream), true, false, &rc)) return rc;
   cudaStream_t st = static_cast<cudaStream_t>(stream);
   const size_t ldA = round_up((size_t)K, 4), ldB = round_up((size_t)N, 4), ldC = ldB;
   const size_t szA = round_up((size_t)M * ldA * 4, 256), szB = round_up((size_t)K * ldB * 4, 256);
@@ -845,14 +880,16 @@ int sgemm_cube_choose_input_scaling(const int64_t* range_a, const int64_t* range
 int sgemm_cube_scaled(sgemm_cube_handle h, int M, int N, int K, const float* A, int64_t lda,
                       const float* B, int64_t ldb, float* C, int64_t ldc, int p_a, int p_b,
                       int scale_exp, int order, void* stream) {
-  if (!h || !A || !B || !C) return SGEMM_CUBE_INVALID_ARG;
+  if (!h) return SGEMM_CUBE_INVALID_ARG;
   int rc = check_gemm_dims(M, N, K, lda, ldb, ldc);
   if (rc) return rc;
+  if (missing_operand(M, N, K, A, A, B, B, C)) return SGEMM_CUBE_INVALID_ARG;
   if (scale_exp < 0 || scale_exp > 24) return SGEMM_CUBE_INVALID_ARG;
   if (order != SGEMM_CUBE_TERMWISE && order != SGEMM_CUBE_ELEMENTWISE) return SGEMM_CUBE_INVALID_ARG;
   if (p_a < -126 || p_a > 126 || p_b < -126 || p_b > 126) return SGEMM_CUBE_INVALID_ARG;
   DeviceGuard g(h->device);
   if (!g.ok) return SGEMM_CUBE_CUDA_ERROR;
+  if (empty_problem(M, N, K, C, ldc, static_cast<cudaStream_t>(stream), false, false, &rc)) return rc;
   cudaStream_t st = static_cast<cudaStream_t>(stream);
   rc = launch_two_phase(h, M, N, K, A, lda, B, ldb, C, ldc, scale_exp, order, st, ldexpf(1.0f, p_a),
                         ldexpf(1.0f, p_b));
@@ -872,9 +909,12 @@ int sgemm_cube_scaled(sgemm_cube_handle h, int M, int N, int K, const float* A, 
 int sgemm_cube_auto_scaled(sgemm_cube_handle h, int M, int N, int K, const float* A, int64_t lda,
                            const float* B, int64_t ldb, float* C, int64_t ldc, int order, void* stream,
                            int* chosen_out) {
-  if (!h || !A || !B || !C) return SGEMM_CUBE_INVALID_ARG;
+  if (!h) return SGEMM_CUBE_INVALID_ARG;
   int rc = check_gemm_dims(M, N, K, lda, ldb, ldc);
   if (rc) return rc;
+  if (missing_operand(M, N, K, A, A, B, B, C)) return SGEMM_CUBE_INVALID_ARG;
+  if (M == 0 || N == 0 || K == 0)
+    return sgemm_cube_scaled(h, M, N, K, A, lda, B, ldb, C, ldc, 0, 0, 11, order, stream);
   int64_t ra[3], rb[3];
   if ((rc = sgemm_cube_hi_exponent_range(h, M, K, A, lda, ra, stream))) return rc;
   if ((rc = sgemm_cube_hi_exponent_range(h, K, N, B, ldb, rb, stream))) return rc;
@@ -1015,10 +1055,11 @@ int static_setup(int device, StaticDeviceState** out) {
 extern "C" int sgemm_cube_unfused_static(int M, int N, int K, const float* A, int64_t lda,
                                          const float* B, int64_t ldb, float* C, int64_t ldc,
                                          int scale_exp, void* stream) {
-  if (!A || !B || !C) return SGEMM_CUBE_INVALID_ARG;
   int rc = check_gemm_dims(M, N, K, lda, ldb, ldc);
   if (rc) return rc;
+  if (missing_operand(M, N, K, A, A, B, B, C)) return SGEMM_CUBE_INVALID_ARG;
   if (scale_exp < 0 || scale_exp > 24) return SGEMM_CUBE_INVALID_ARG;
+  if (empty_problem(M, N, K, C, ldc, static_cast<cudaStream_t>(stream), false, false, &rc)) return rc;
   // Same layout as the workspace of sgemm_cube_unfused, carved out of the fixed array.
   const size_t ldA16 = round_up((size_t)K, 8), ldB16 = round_up((size_t)N, 8);
   const size_t ldD = round_up((size_t)N, 4);

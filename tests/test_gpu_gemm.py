@@ -344,7 +344,8 @@ def test_argument_errors(handle):
                                        kw.get("ldb", 8), kw.get("C", p(C)), kw.get("ldc", 8),
                                        kw.get("s", 11), kw.get("order", 0), None)
     assert call() == binding.OK
-    assert call(M=0) == binding.INVALID_ARG
+    assert call(M=-1) == binding.INVALID_ARG
+    assert call(M=0) == binding.OK                           # empty problems are valid
     assert call(K=-1) == binding.INVALID_ARG
     assert call(lda=15) == binding.INVALID_ARG
     assert call(ldc=7) == binding.INVALID_ARG
@@ -401,3 +402,41 @@ def test_kernel_timing_queries(handle):
         assert n == 128 and 0 < mean < 50
     finally:
         handle.sgemm_cube_set_option(binding.OPT_TIME_KERNEL, 0)
+
+
+@pytest.mark.parametrize("shape", [(0, 5, 7), (5, 0, 7), (5, 8, 0), (0, 0, 0)])
+def test_empty_problems(handle, shape):
+    # No output elements: nothing happens.  Empty inner dimension: the empty sum, C = 0, as the
+    # oracle's loops give.
+    M, N, K = shape
+    f32 = dict(dtype=torch.float32, device="cuda:0")
+    A, B = torch.ones((M, K), **f32), torch.ones((K, N), **f32)
+    want = oracle.sgemm_cube(np.ones((M, K), np.float32), np.ones((K, N), np.float32), 11, T, 64) \
+        if M and N else np.zeros((M, N), np.float32)
+    calls = [lambda C: handle.sgemm_cube(A, B, C, 11, T), lambda C: handle.sgemm_cube(A, B, C, 11, E),
+             lambda C: handle.sgemm_cube_unfused(A, B, C, 11, T),
+             lambda C: handle.sgemm_cube_four_term(A, B, C, 11),
+             lambda C: handle.sgemm_cube_scaled(A, B, C, 3, -2, 11, T),
+             lambda C: handle.sgemm_cube_auto_scaled(A, B, C, T),
+             lambda C: binding.sgemm_cube_unfused_static(A, B, C, 11)]
+    for call in calls:
+        C = torch.full((M, N), 7.0, **f32)
+        call(C)
+        assert handle.sgemm_cube_check()[0] == 0
+        assert np.array_equal(C.cpu().numpy(), want)
+    f16 = dict(dtype=torch.float16, device="cuda:0")
+    Ah, Bh = torch.ones((M, K), **f16), torch.ones((K, N), **f16)
+    D = torch.full((M, N), 7.0, **f32)
+    handle.sgemm_cube_hgemm(Ah, Bh, D, accumulate=True)
+    assert torch.all(D == 7.0)                              # nothing to add
+    handle.sgemm_cube_hgemm(Ah, Bh, D)
+    assert np.array_equal(D.cpu().numpy(), want)
+    handle.sgemm_cube_presplit(Ah, Ah.clone(), Bh, Bh.clone(), D, 11, T)
+    assert np.array_equal(D.cpu().numpy(), want)
+    handle.sgemm_cube_split(A, Ah, Ah.clone(), 11)          # empty split: no-op
+    Ch = torch.full((M, N), 7.0).pin_memory() if M * N else torch.empty((M, N))
+    handle.sgemm_cube_host(torch.ones((M, K)), torch.ones((K, N)), Ch, 11, T)
+    assert np.array_equal(Ch.numpy(), want)
+    with pytest.raises(binding.SgemmCubeError):
+        load = binding.load()
+        binding._check(load.sgemm_cube(handle._h, -1, 4, 4, None, 4, None, 4, None, 4, 11, T, None), "neg")

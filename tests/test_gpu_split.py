@@ -96,8 +96,9 @@ def test_split_rejects_bad_arguments(handle):
         handle.sgemm_cube_split(X, hi, hi.clone(), 25)
     assert e.value.status == binding.INVALID_ARG
     lib = binding.load()
-    assert lib.sgemm_cube_split(handle._h, 0, 8, X.data_ptr(), 8, hi.data_ptr(), hi.data_ptr(), 8, 11,
+    assert lib.sgemm_cube_split(handle._h, -1, 8, X.data_ptr(), 8, hi.data_ptr(), hi.data_ptr(), 8, 11,
                                 None) == binding.INVALID_ARG
+    assert lib.sgemm_cube_split(handle._h, 0, 8, None, 8, None, None, 8, 11, None) == binding.OK   # empty
     assert lib.sgemm_cube_split(handle._h, 4, 8, X.data_ptr(), 4, hi.data_ptr(), hi.data_ptr(), 8, 11,
                                 None) == binding.INVALID_ARG
     assert lib.sgemm_cube_split(handle._h, 4, 8, None, 8, hi.data_ptr(), hi.data_ptr(), 8, 11,

@@ -52,5 +52,9 @@ def test_static_scratch_variant_rejects_what_does_not_fit():
     torch.cuda.synchronize()
     assert torch.all(C == 3.0)            # nothing was enqueued
     lib = binding.load()
-    assert lib.sgemm_cube_unfused_static(0, 8, 8, A.data_ptr(), 8, B.data_ptr(), 8, C.data_ptr(), 8,
+    assert lib.sgemm_cube_unfused_static(-1, 8, 8, A.data_ptr(), 8, B.data_ptr(), 8, C.data_ptr(), 8,
                                          11, None) == binding.INVALID_ARG
+    assert lib.sgemm_cube_unfused_static(0, 8, 8, A.data_ptr(), 8, B.data_ptr(), 8, C.data_ptr(), 8,
+                                         11, None) == binding.OK            # empty: nothing to do
+    torch.cuda.synchronize()
+    assert torch.all(C == 3.0)

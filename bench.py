@@ -6,7 +6,7 @@
 One "step" is one pass of the whole hot path over one batch of synthetic input: a single call of
 the `sgemm_cube` entry point with its default options (operand split, three FP16 tensor-core
 products and the FP32 reconstruction; at this size the library splits both operands once with the
-split kernel and forms the products in one tensor-core kernel: three launches per step) on
+split kernel and forms the products in one tensor-core kernel: two launches per step) on
 M = N = K = 8192 FP32 matrices whose entries are
 (+/-) u * 2^e, u uniform in [1, 2), e a uniform integer in [-10, 10], with s = 11 and termwise
 accumulation.  The metric is FP32-equivalent TFLOP/s = 2 M N K / t.
@@ -360,7 +360,7 @@ def main():
             "warmup": warmup, "ms_per_step": ms_per_step, "higher_is_better": True,
             "scaling": "weak", "vs_baseline": None, "dtype": "f16 products, f32 accumulate",
             "data": "synthetic",
-            "config": {"workload": WORKLOAD, "entry_point": "sgemm_cube, strategy %s: split kernel x2 + three-product "
+            "config": {"workload": WORKLOAD, "entry_point": "sgemm_cube, strategy %s: split kernel (both operands, one launch) + three-product "
                                       "tensor-core kernel per step" % args.strategy
                        if args.strategy != "fused" else "sgemm_cube, strategy fused: one kernel per step",
                        "l2": "inputs (512 MiB) larger than L2; no flush",

@@ -219,7 +219,7 @@ int sgemm_cube_host(sgemm_cube_handle h, int M, int N, int K,
  * It exists to measure what dropping that term costs; it is not part of the paper's method.
  * Termwise only: each stream is summed in k-blocks (SGEMM_CUBE_OPT_TERMWISE_K_BLOCK) and
  *   C = S_hh + (2^-s S_x + 2^-2s S_ll),
- * the small terms combined first.  Runs as: two split launches, one FP16 GEMM pass lo_A lo_B into
+ * the small terms combined first.  Runs as: the split of both operands, one FP16 GEMM pass lo_A lo_B into
  * the handle's workspace, the three-product kernel writing its raw sums, one reduction kernel.
  * Arguments, layouts and alignment-free inputs as sgemm_cube_unfused.  Workspace:
  * 4 bytes x (M K + K N) + 12 bytes x M N, rounded up, grown with cudaMalloc on first use.

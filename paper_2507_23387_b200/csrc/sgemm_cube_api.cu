@@ -210,6 +210,35 @@ int launch_split(sgemm_cube_ctx* h, int rows, int cols, const float* X, int64_t 
   return cudaGetLastError() == cudaSuccess ? SGEMM_CUBE_OK : SGEMM_CUBE_CUDA_ERROR;
 }
 
+// Split A (M x K) and B (K x N) of one product: one launch when both take the vector path.
+int launch_split_pair(sgemm_cube_ctx* h, int M, int N, int K, const float* A, int64_t lda, uint16_t* Ahi,
+                      uint16_t* Alo, int64_t ldA16, const float* B, int64_t ldb, uint16_t* Bhi,
+                      uint16_t* Blo, int64_t ldB16, int s, cudaStream_t st, float pre_a = 1.0f,
+                      float pre_b = 1.0f) {
+  const bool vec_a = (K % 8 == 0) && aligned16(A) && (lda % 4 == 0) && aligned16(Ahi) && aligned16(Alo) &&
+                     (ldA16 % 8 == 0);
+  const bool vec_b = (N % 8 == 0) && aligned16(B) && (ldb % 4 == 0) && aligned16(Bhi) && aligned16(Blo) &&
+                     (ldB16 % 8 == 0);
+  if (!vec_a || !vec_b) {
+    int rc = launch_split(h, M, K, A, lda, Ahi, Alo, ldA16, s, st, pre_a);
+    if (rc) return rc;
+    return launch_split(h, K, N, B, ldb, Bhi, Blo, ldB16, s, st, pre_b);
+  }
+  const long long items_a = (long long)M * (K / 8), items_b = (long long)K * (N / 8);
+  long long blocks = (items_a + items_b + 255) / 256;
+  const long long cap = (long long)h->sm_count * 16;
+  if (blocks > cap) blocks = cap;
+  if (blocks < 2) blocks = 2;
+  long long blocks_a = (long long)((double)blocks * (double)items_a / (double)(items_a + items_b) + 0.5);
+  if (blocks_a < 1) blocks_a = 1;
+  if (blocks_a > blocks - 1) blocks_a = blocks - 1;
+  const sgc::SplitOperand a{M, K, A, lda, Ahi, Alo, ldA16, pre_a};
+  const sgc::SplitOperand b{K, N, B, ldb, Bhi, Blo, ldB16, pre_b};
+  sgc::split2_vec8_kernel<<<(unsigned)blocks, 256, 0, st>>>(a, b, s, (unsigned)blocks_a);
+  h->launches++;
+  return cudaGetLastError() == cudaSuccess ? SGEMM_CUBE_OK : SGEMM_CUBE_CUDA_ERROR;
+}
+
 // FP16-operand tensor-core GEMM launch, NTERMS = 1 (lo pointers unused) or 3.
 template <int NTERMS>
 int launch_tc_gemm(sgemm_cube_ctx* h, int M, int N, int K, const uint16_t* Ahi, const uint16_t* Alo,
@@ -345,8 +374,9 @@ int launch_two_phase(sgemm_cube_ctx* h, int M, int N, int K, const float* A, int
   uint16_t* Alo = reinterpret_cast<uint16_t*>(w + szA);
   uint16_t* Bhi = reinterpret_cast<uint16_t*>(w + 2 * szA);
   uint16_t* Blo = reinterpret_cast<uint16_t*>(w + 2 * szA + szB);
-  if ((rc = launch_split(h, M, K, A, lda, Ahi, Alo, (int64_t)ldA16, s, st, pre_a))) return rc;
-  if ((rc = launch_split(h, K, N, B, ldb, Bhi, Blo, (int64_t)ldB16, s, st, pre_b))) return rc;
+  if ((rc = launch_split_pair(h, M, N, K, A, lda, Ahi, Alo, (int64_t)ldA16, B, ldb, Bhi, Blo, (int64_t)ldB16, s,
+                              st, pre_a, pre_b)))
+    return rc;
   const int kblock = (order == SGEMM_CUBE_TERMWISE) ? h->kblock_termwise : h->kblock_elementwise;
   const int slot = (int)(h->ev_calls % sgemm_cube_ctx::kTimedCalls);
   if (h->time_kernel) cudaEventRecord(h->ev_ring[2 * slot], st);
@@ -601,8 +631,9 @@ int sgemm_cube_unfused(sgemm_cube_handle h, int M, int N, int K, const float* A,
   float* Dx = reinterpret_cast<float*>(w + 2 * szA + 2 * szB + szD);
   const float inv = ldexpf(1.0f, -scale_exp);
   const int kb = h->kblock_termwise;
-  if ((rc = launch_split(h, M, K, A, lda, Ahi, Alo, (int64_t)ldA16, scale_exp, st))) return rc;
-  if ((rc = launch_split(h, K, N, B, ldb, Bhi, Blo, (int64_t)ldB16, scale_exp, st))) return rc;
+  if ((rc = launch_split_pair(h, M, N, K, A, lda, Ahi, Alo, (int64_t)ldA16, B, ldb, Bhi, Blo, (int64_t)ldB16,
+                              scale_exp, st)))
+    return rc;
   if ((rc = launch_tc_gemm<1>(h, M, N, K, Ahi, nullptr, ldA16, Bhi, nullptr, ldB16, Dhh, ldD, 0, 0, kb, 1.f, st))) return rc;
   if ((rc = launch_tc_gemm<1>(h, M, N, K, Alo, nullptr, ldA16, Bhi, nullptr, ldB16, Dx, ldD, 0, 0, kb, 1.f, st))) return rc;
   if ((rc = launch_tc_gemm<1>(h, M, N, K, Ahi, nullptr, ldA16, Blo, nullptr, ldB16, Dx, ldD, 1, 0, kb, 1.f, st))) return rc;
@@ -641,8 +672,9 @@ int sgemm_cube_four_term(sgemm_cube_handle h, int M, int N, int K, const float* 
   uint16_t* Blo = reinterpret_cast<uint16_t*>(w + 2 * szA + szB);
   float* Dll = reinterpret_cast<float*>(w + 2 * szA + 2 * szB);
   const int kb = h->kblock_termwise;
-  if ((rc = launch_split(h, M, K, A, lda, Ahi, Alo, (int64_t)ldA16, scale_exp, st))) return rc;
-  if ((rc = launch_split(h, K, N, B, ldb, Bhi, Blo, (int64_t)ldB16, scale_exp, st))) return rc;
+  if ((rc = launch_split_pair(h, M, N, K, A, lda, Ahi, Alo, (int64_t)ldA16, B, ldb, Bhi, Blo, (int64_t)ldB16,
+                              scale_exp, st)))
+    return rc;
   if ((rc = launch_tc_gemm<1>(h, M, N, K, Alo, nullptr, ldA16, Blo, nullptr, ldB16, Dll, ldD, 0, 0, kb, 1.f, st)))
     return rc;
   return launch_tc_gemm<3>(h, M, N, K, Ahi, Alo, (int64_t)ldA16, Bhi, Blo, (int64_t)ldB16, C, ldc, 0,

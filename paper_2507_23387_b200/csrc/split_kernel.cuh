@@ -65,6 +65,53 @@ split_vec8_kernel(int rows, int cols, const float* __restrict__ X, long long ldx
   }
 }
 
+// Both operands of a product in one launch (same arithmetic as split_vec8_kernel; saves a launch
+// and its ramp-up and tail, which count for mid-sized problems).  The first `blocks_a` CTAs take
+// operand a, the rest operand b; the host splits the grid in proportion to the element counts.
+struct SplitOperand {
+  int rows, cols;
+  const float* X;
+  long long ldx;
+  uint16_t* hi;
+  uint16_t* lo;
+  long long ldh;
+  float pre;
+};
+__device__ __forceinline__ void split_vec8_items(const SplitOperand& a, float scale, long long first,
+                                                 long long stride) {
+  const bool prescale = a.pre != 1.0f;
+  const long long items_per_row = a.cols >> 3;
+  const long long total = (long long)a.rows * items_per_row;
+  for (long long it = first; it < total; it += stride) {
+    const long long r = it / items_per_row;
+    const long long c = (it - r * items_per_row) << 3;
+    const float4* src = reinterpret_cast<const float4*>(a.X + r * a.ldx + c);
+    float4 u = __ldg(src);
+    float4 v = __ldg(src + 1);
+    if (prescale) {
+      u.x = __fmul_rn(u.x, a.pre); u.y = __fmul_rn(u.y, a.pre); u.z = __fmul_rn(u.z, a.pre); u.w = __fmul_rn(u.w, a.pre);
+      v.x = __fmul_rn(v.x, a.pre); v.y = __fmul_rn(v.y, a.pre); v.z = __fmul_rn(v.z, a.pre); v.w = __fmul_rn(v.w, a.pre);
+    }
+    uint4 h, l;
+    split_two(u.x, u.y, scale, h.x, l.x);
+    split_two(u.z, u.w, scale, h.y, l.y);
+    split_two(v.x, v.y, scale, h.z, l.z);
+    split_two(v.z, v.w, scale, h.w, l.w);
+    *reinterpret_cast<uint4*>(a.hi + r * a.ldh + c) = h;
+    *reinterpret_cast<uint4*>(a.lo + r * a.ldh + c) = l;
+  }
+}
+__global__ void __launch_bounds__(256)
+split2_vec8_kernel(SplitOperand a, SplitOperand b, int scale_exp, unsigned int blocks_a) {
+  const float scale = pow2f(scale_exp);
+  if (blockIdx.x < blocks_a)
+    split_vec8_items(a, scale, (long long)blockIdx.x * blockDim.x + threadIdx.x,
+                     (long long)blocks_a * blockDim.x);
+  else
+    split_vec8_items(b, scale, (long long)(blockIdx.x - blocks_a) * blockDim.x + threadIdx.x,
+                     (long long)(gridDim.x - blocks_a) * blockDim.x);
+}
+
 // General path: any alignment, any cols.
 __global__ void __launch_bounds__(256)
 split_scalar_kernel(int rows, int cols, const float* __restrict__ X, long long ldx,

@@ -72,11 +72,12 @@ enum {
   SGEMM_CUBE_OPT_ELEMENTWISE_K_BLOCK = 1,
   /* 1: run the tensor-core kernels as clusters of two CTAs that share one
    * tcgen05.mma.cta_group::2 (256 x 256 tile per pair, each CTA loading half of the B tile);
-   * 0 (default): one CTA per 128 x 256 tile; 2: pairs when the problem has at least four waves
-   * of pair tiles.  Same arithmetic, bit-identical results either way as long as split-K (below,
-   * single CTAs only) does not apply.  (Pairs halve the B-tile traffic and are the faster mode
-   * for k-blocks of 512 and more; at the default k-block of 128 the more frequent TMEM drains
-   * cost them more than they save.) */
+   * 0: one CTA per 128 x 256 tile; 2 (default): the library chooses: pairs for the kernels that
+   * read FP16 words (two-phase sgemm_cube, sgemm_cube_presplit, sgemm_cube_hgemm, ...) whenever
+   * M > 128 and split-K (below, single CTAs only) does not apply, single CTAs for the fused
+   * converter kernel.  Same arithmetic, bit-identical results either way as long as split-K does
+   * not apply.  (Pairs pull two thirds of the bytes of single CTAs from L2 into the SMs, which is
+   * what bounds this kernel: 458 against 439 TFLOP/s at 8192^3, 407 against 378 at 4096^3.) */
   SGEMM_CUBE_OPT_CTA_PAIR = 2,
   /* How sgemm_cube computes (same arithmetic; same bracketing and bit-identical results except
    * where split-K, which only the two-phase strategy uses, re-brackets the k-block sums):

@@ -372,7 +372,7 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA0, const __grid_constant__
     // "TMEM region drained": arrive on the leader's barrier (the peer does so remotely).
     auto arrive_tempty = [&](int r) {
       if (!PAIR || leader) mbar_arrive(&tempty_bar[r]);
-      else mbar_arrive_cluster(mapa_u32(smem_u32(&tempty_bar[r]), 0));
+      else mbar_arrive_cluster_relaxed(mapa_u32(smem_u32(&tempty_bar[r]), 0));
     };
     for (int unit = first_tile; unit < num_units && ok; unit += tile_stride) {
       int tm, tn, kb0, kb1, slice;
@@ -385,6 +385,7 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA0, const __grid_constant__
           SGC_T0();
           if (!wait_tfull(r_main)) { ok = false; break; }
           SGC_TADD(6, blockIdx.x == 0 && threadIdx.x == 0);
+          SGC_TADD(13, blockIdx.x == 1 && threadIdx.x == 0);
         }
         SGC_T0();
         if (with_x && !wait_tfull(1)) { ok = false; break; }
@@ -414,6 +415,7 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA0, const __grid_constant__
         }
         tc_fence_before_sync();
         __syncwarp();
+        SGC_TADD(15, blockIdx.x == 1 && threadIdx.x == 0);
         if (lane == 0) {
           arrive_tempty(r_main);
           if (with_x) arrive_tempty(1);
@@ -421,6 +423,7 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA0, const __grid_constant__
         drains[r_main]++;
         if (with_x) drains[1]++;
         SGC_TADD(7, blockIdx.x == 0 && threadIdx.x == 0);
+        SGC_TADD(14, blockIdx.x == 1 && threadIdx.x == 0);
       }
       if (!ok) break;
       SGC_T0();
@@ -611,7 +614,7 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA0, const __grid_constant__
             return true;
           };
           // hi_A hi_B (or the single product) of one stage into the main region; frees the stage.
-          auto issue_main = [&](uint32_t st, uint32_t i, bool first_kb) -> bool {
+          auto issue_main = [&](uint32_t st, uint32_t i, bool first_kb, bool release = true) -> bool {
             if (!main_ready) {
               SGC_T0();
               if (!wait(&tempty_bar[r_main], (fills[r_main] & 1) ^ 1, kErrMmaTmemEmptyWait)) return false;
@@ -627,7 +630,8 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA0, const __grid_constant__
               const uint64_t db = desc(b_hi + 128 * j, b_desc_hi);
               mma(d_main, da, db, (first_kb && j == 0) ? 0u : 1u);
             }
-            commit_both(&empty_bar[i % STAGES]);   // the stage may be refilled once these MMAs retire
+            // the stage may be refilled once these MMAs retire
+            if (release) commit_both(&empty_bar[i % STAGES]);
             return true;
           };
           int kb = kb_begin;
@@ -635,7 +639,7 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA0, const __grid_constant__
 #ifdef SGC_KLOOK
           constexpr int kLook = SGC_KLOOK;
 #else
-          constexpr int kLook = ((PAIR ? 3 : 2) * 32 + BK - 1) / BK;
+          constexpr int kLook = (((PAIR && FUSED) ? 3 : 2) * 32 + BK - 1) / BK;
 #endif
           if (NTERMS == 3 && p.order == 0 && kb + kLook <= kb_end) {
             // Start of a termwise k-block: the correction products of the first kLook stages go
@@ -650,16 +654,35 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA0, const __grid_constant__
             kb += kLook;
             it += kLook;
           }
+          bool handed_over = false;
           for (; kb < kb_end && ok; ++kb, ++it) {
             uint32_t st;
             const bool first_kb = (kb == kb_begin);
+#ifndef SGC_NO_TAIL_SWAP
+            if (NTERMS == 3 && p.order == 0 && kb == kb_end - 1 && !first_kb) {
+              // Last stage of a termwise k-block of two or more stages: hi*hi first, so that
+              // region 0 goes to the accumulate warps eight MMAs earlier; this stage's correction
+              // products and those of the next block's first stage then run while it is drained.
+              // The order inside each chain is unchanged.
+              ok = stage_ready(it, st) && issue_main(st, it, false, /*release*/ false);
+              if (!ok) break;
+              commit_both(&tfull_bar[r_main]);
+              fills[r_main]++;
+              handed_over = true;
+              ok = issue_cross(st, false);
+              commit_both(&empty_bar[it % STAGES]);
+              continue;
+            }
+#endif
             ok = stage_ready(it, st) && (NTERMS != 3 || issue_cross(st, first_kb)) &&
                  issue_main(st, it, first_kb);
           }
           if (!ok) break;
           // Hand the finished region(s) to the accumulate warps.
-          commit_both(&tfull_bar[r_main]);
-          fills[r_main]++;
+          if (!handed_over) {
+            commit_both(&tfull_bar[r_main]);
+            fills[r_main]++;
+          }
           if (NTERMS == 3 && (p.order == 1 || c == unit_chunks - 1)) {
             commit_both(&tfull_bar[1]);
             fills[1]++;

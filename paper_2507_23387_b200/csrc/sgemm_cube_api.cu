@@ -52,7 +52,7 @@ struct sgemm_cube_ctx {
   long long launches = 0;
   int kblock_termwise = 128;
   int kblock_elementwise = 64;
-  int cta_pair = 0;            // 0/1: never/always 2-CTA clusters (cta_group::2); 2: by problem size
+  int cta_pair = 2;            // 0/1: never/always 2-CTA clusters (cta_group::2); 2: see use_pair
   int strategy = 0;            // sgemm_cube: 0 auto, 1 fused kernel, 2 split kernel + 3-product kernel
   int time_kernel = 0;         // record events around the tensor-core kernel of sgemm_cube
   static constexpr int kTimedCalls = 128;           // event pairs kept (most recent calls)
@@ -116,12 +116,15 @@ int set_kernel_attrs(sgemm_cube_ctx* h) {
   return SGEMM_CUBE_OK;
 }
 
-// 2-CTA clusters pay off once there are enough 256 x 256 pair tiles to keep every SM pair busy
-// for several waves; below that the finer 128 x 256 tiles balance better.
-bool use_pair(const sgemm_cube_ctx* h, int M, int N) {
+// 2-CTA clusters (each CTA loads half of the B tile: two thirds of the L2 -> SM traffic of single
+// CTAs) measured faster than single CTAs for the TMA-fed kernels from 512^3 up (e.g. 4096^3: 407
+// against 378, 8192^3: 458 against 439 TFLOP/s); by default they are used whenever the problem has
+// more than one 128-row block.  The converter-fed kernel is slower in pairs (172 against 193) and
+// only uses them when asked to.
+bool use_pair(const sgemm_cube_ctx* h, int M, int N, bool fused) {
+  (void)N;
   if (h->cta_pair != 2) return h->cta_pair == 1;
-  const long long pair_tiles = (long long)((M + 255) / 256) * ((N + 255) / 256);
-  return pair_tiles >= 4LL * (h->sm_count / 2);
+  return !fused && M > sgc::kBM;
 }
 
 // Launch one tensor-core kernel: a persistent grid of single CTAs, or of 2-CTA clusters (PAIR).
@@ -284,8 +287,9 @@ int launch_tc_gemm(sgemm_cube_ctx* h, int M, int N, int K, const uint16_t* Ahi, 
   // Split-K: when the tiles would leave more than half of the SMs idle and k is long, cut the k
   // range into slices (whole k-blocks) so that tiles x slices fills the machine; a reduction
   // kernel adds the slices' sums.
-  const bool pair = use_pair(h, M, N) && !Dll;
-  if (NTERMS == 3 && h->split_k && !pair) {
+  bool pair = use_pair(h, M, N, false) && !Dll;
+  // Split-K runs on single CTAs; with the pair mode left to the library it takes precedence.
+  if (NTERMS == 3 && h->split_k && (!pair || h->cta_pair == 2)) {
     const int tiles = ((M + sgc::kBM - 1) / sgc::kBM) * ((N + sgc::kBN - 1) / sgc::kBN);
     const int num_kb = (K + Cfg::BK - 1) / Cfg::BK;
     const int chunks = (num_kb + p.kchunk_blocks - 1) / p.kchunk_blocks;
@@ -299,6 +303,7 @@ int launch_tc_gemm(sgemm_cube_ctx* h, int M, int N, int K, const uint16_t* Ahi, 
       const size_t pstride = round_up((size_t)M * ldp, 64);
       const size_t need = (size_t)slices * pstride * 4 * (order == SGEMM_CUBE_TERMWISE ? 2 : 1);
       if (slices >= 2 && grow(&h->part_ws, &h->part_ws_bytes, need) == SGEMM_CUBE_OK) {
+        pair = false;
         p.ksplit = slices;
         p.kslice_blocks = chunks_per_slice * p.kchunk_blocks;
         p.Phh = static_cast<float*>(h->part_ws);
@@ -356,7 +361,7 @@ int launch_fused(sgemm_cube_ctx* h, int M, int N, int K, const float* A, int64_t
   p.ksplit = 1; p.kslice_blocks = 0; p.Phh = nullptr; p.Px = nullptr; p.pstride = 0; p.ldp = 0;
   CUtensorMap unused;
   memset(&unused, 0, sizeof(unused));
-  return use_pair(h, M, N) ? launch_tc_kernel<3, true, true>(h, M, N, unused, unused, unused, unused, p, st)
+  return use_pair(h, M, N, true) ? launch_tc_kernel<3, true, true>(h, M, N, unused, unused, unused, unused, p, st)
                            : launch_tc_kernel<3, true, false>(h, M, N, unused, unused, unused, unused, p, st);
 }
 

@@ -100,6 +100,9 @@ struct TcGemmParams {
   long long ldp;
 };
 
+#ifndef SGC_PAIR_GROUP
+#define SGC_PAIR_GROUP 8
+#endif
 #ifndef SGC_BK3
 #define SGC_BK3 64
 #endif
@@ -332,7 +335,7 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA0, const __grid_constant__
   const int first_tile = PAIR ? (int)(blockIdx.x >> 1) : (int)blockIdx.x;
   const int tile_stride = PAIR ? (int)(gridDim.x >> 1) : (int)gridDim.x;
   auto tile_rc = [&](int tile, int& tm, int& tn) {     // tm in units of 128 rows, tn of 256 columns
-    tile_coords(tile, num_m, num_n, tm, tn, PAIR ? 8 : 16);
+    tile_coords(tile, num_m, num_n, tm, tn, PAIR ? SGC_PAIR_GROUP : 16);
     if (PAIR) tm = tm * 2 + (int)cta_rank;
   };
   const int num_kb = (p.K + BK - 1) / BK;                      // pipeline stages per tile

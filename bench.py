@@ -38,7 +38,7 @@ UNIT = "TFLOP/s"
 # DRAM traffic of one launch of the dominant kernel (the three-product tensor-core kernel) at this
 # workload: dram__bytes_read.sum + dram__bytes_write.sum of the full-size one-pass ncu capture
 # summarised in profiles/three_product_kernel_8192_cubed.md.
-KERNEL_DRAM_BYTES_PER_LAUNCH = 2277921024 + 255401984
+KERNEL_DRAM_BYTES_PER_LAUNCH = 3102864640 + 259538944
 
 
 def measured_peaks():

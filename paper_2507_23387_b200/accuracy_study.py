@@ -11,6 +11,11 @@ Eq. err, mean over seeds):
                                                                       (Fig. mkn_error)
   dropped term     three-term SGEMM-cube against the four-term variant that keeps lo_A lo_B
                    (the term Eq. ll_bound bounds), against k
+  adversarial      the max-norm study on constructed inputs that Sec. 6.2 and Sec. 7 name as
+                   missing: products that cancel down to a fraction c of |A||B|, and entries whose
+                   residuals all have the largest size and the same sign; reported is the largest
+                   componentwise error max |C - C64| / (|A||B|) in units of u_32 = 2^-24 (the
+                   quantity Eq. main_bound bounds) and the largest relative error of an entry
 
 Everything runs through the library's C ABI (`sgemm_cube`, `sgemm_cube_split`,
 `sgemm_cube_hgemm`, `sgemm_cube_four_term`); the FP64 reference and the FP32 baseline are torch matmuls on the device.
@@ -142,6 +147,42 @@ def dropped_term_sweep(h, ks=(8, 32, 128, 512, 2048, 8192), mn=1024, seeds=5, sc
     return rows
 
 
+def adversarial_sweep(h, mn=1024, seeds=3, scale_exp=11, device="cuda:0",
+                      cancellations=(1.0, 2.0 ** -6, 2.0 ** -12, 2.0 ** -18), k_cancel=1024,
+                      ks_coherent=(16, 256, 4096)):
+    """Constructed inputs (inputs.cancellation_pair, inputs.coherent_residuals).  Per case and
+    method: eta = max |C - C64| / (|A||B|) in units of 2^-24 over all seeds, and the largest
+    relative error of an entry (cancellation cases)."""
+    methods = (("termwise", lambda A, B, C: h.sgemm_cube(A, B, C, scale_exp, binding.TERMWISE)),
+               ("elementwise", lambda A, B, C: h.sgemm_cube(A, B, C, scale_exp, binding.ELEMENTWISE)),
+               ("four_term", lambda A, B, C: h.sgemm_cube_four_term(A, B, C, scale_exp)),
+               ("fp32_gemm", lambda A, B, C: C.copy_(_fp32_gemm(A, B))))
+    cases = [("cancel c=2^%d" % round(torch.log2(torch.tensor(c)).item()), k_cancel,
+              lambda seed, c=c: inputs.cancellation_pair(seed, mn, mn, k_cancel, c)) for c in cancellations]
+    cases += [("coherent residuals k=%d" % k, k,
+               lambda seed, k=k: (inputs.coherent_residuals(seed, (mn, k), 0),
+                                  inputs.coherent_residuals(seed, (k, mn), 1))) for k in ks_coherent]
+    rows = []
+    C = torch.empty((mn, mn), device=device)
+    for name, K, make in cases:
+        r = {"case": name, "k": K, "bound_first_order": float(K + 14)}
+        for seed in range(seeds):
+            A, B = (torch.from_numpy(x).to(device) for x in make(seed))
+            C64 = _reference(A, B)
+            AB = A.double().abs() @ B.double().abs()
+            for mname, call in methods:
+                call(A, B, C)
+                err = (C.double() - C64).abs()
+                r[mname + "_eta"] = max(r.get(mname + "_eta", 0.0), float((err / AB).max()) * 2.0 ** 24)
+                rel = float((err / C64.abs().clamp_min(1e-300)).max())
+                r[mname + "_maxrel"] = max(r.get(mname + "_maxrel", 0.0), rel)
+        rows.append(r)
+    status, detail = h.sgemm_cube_check()
+    if status != 0:
+        raise RuntimeError("device error %s" % hex(detail))
+    return rows
+
+
 def _table(rows, key, cols):
     lines = ["| %s | %s |" % (key, " | ".join(cols)), "|" + "---|" * (len(cols) + 1)]
     for r in rows:
@@ -170,7 +211,8 @@ def main():
     res = {"symmetric": sym, "nonnegative": pos, "vs_mn": size_sweep(h, mn, args.seeds),
            "vs_k": size_sweep(h, ks, args.seeds), "vs_all": size_sweep(h, alls, args.seeds),
            "dropped_term": dropped_term_sweep(h, (8, 512) if args.quick else (8, 32, 128, 512, 2048, 8192),
-                                              seeds=args.seeds)}
+                                              seeds=args.seeds),
+           "adversarial": adversarial_sweep(h, 512 if args.quick else 1024, 1 if args.quick else 3)}
     h.destroy()
     if args.json:
         print(json.dumps(res))
@@ -188,6 +230,13 @@ def main():
     print("\n## Three-term against four-term (low-low product kept), m = n = 1024, U[-1, 1), s_b = 11\n")
     print(_table(res["dropped_term"], "k", ["three_term_frob", "four_term_frob", "three_term_cw",
                                             "four_term_cw"]))
+    print("\n## Constructed inputs: largest componentwise error in units of 2^-24 "
+          "(first-order form of Eq. main_bound: k + 14), m = n = 1024, s_b = 11\n")
+    print(_table(res["adversarial"], "case", ["bound_first_order", "termwise_eta", "elementwise_eta",
+                                              "four_term_eta", "fp32_gemm_eta"]))
+    print("\n## Constructed inputs: largest relative error of an entry\n")
+    print(_table(res["adversarial"], "case", ["termwise_maxrel", "elementwise_maxrel", "four_term_maxrel",
+                                              "fp32_gemm_maxrel"]))
 
 
 if __name__ == "__main__":

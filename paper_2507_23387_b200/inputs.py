@@ -102,6 +102,33 @@ def make_pair(kind: str, seed: int, M: int, N: int, K: int):
     raise ValueError("unknown workload kind: %r" % (kind,))
 
 
+# ---- constructed (adversarial) inputs for the max-norm study the paper names as missing (Sec. 6.2,
+#      Sec. 7): no randomness in their structure, only in the values the structure is built from.
+
+def cancellation_pair(seed: int, M: int, N: int, K: int, c: float):
+    """(A, B) whose product cancels down to a fraction ~c of |A||B|:
+    A = [X, -X], B = [Y; Y + c Z] with X, Y, Z uniform on [-1, 1), so that A B = -c X Z while
+    |A||B| ~ 2 |X||Y|.  K must be even."""
+    assert K % 2 == 0
+    X = uniform_pm1(seed, (M, K // 2), 0)
+    Y = uniform_pm1(seed, (K // 2, N), 1)
+    Z = uniform_pm1(seed, (K // 2, N), 2)
+    A = np.concatenate([X, -X], axis=1)
+    B = np.concatenate([Y, (Y + np.float32(c) * Z).astype(np.float32)], axis=0)
+    return np.ascontiguousarray(A), np.ascontiguousarray(B)
+
+
+def coherent_residuals(seed: int, shape, stream: int = 0) -> np.ndarray:
+    """Positive entries just under half a unit in the 11th place above an 11-bit value, all on the
+    same side: x = g + 2^-11 - 2^-22 with g on the 11-bit grid in [1, 1.125).  Every entry then
+    carries a residual of (nearly) the largest relative size, 2^-11, and of the same sign, so
+    whatever a method does with residual products adds up along k instead of averaging out."""
+    shape, n = _shape_n(shape)
+    bits = (raw_u64(seed, stream, n) >> np.uint64(57)).astype(np.float64)      # 7 random bits
+    x = 1.0 + bits * 2.0 ** -10 + 2.0 ** -11 - 2.0 ** -22
+    return x.astype(np.float32).reshape(shape)
+
+
 def device_normal(seed: int, shape, device="cuda:0"):
     """i.i.d. N(0, 1) FP32 generated on the device with a seeded torch generator, for the
     full-size workloads where host generation would dominate the run."""

@@ -75,3 +75,20 @@ def test_dropped_term_sweep(handle):
     assert 0.8 < rows[2048]["four_term_frob"] / rows[2048]["three_term_frob"] < 1.05
     for r in rows.values():
         assert r["four_term_cw"] <= 2 * r["k"] * 2.0 ** -24 and r["three_term_cw"] <= 2 * r["k"] * 2.0 ** -24
+
+
+def test_adversarial_sweep_stays_inside_the_componentwise_bound(handle):
+    rows = accuracy_study.adversarial_sweep(handle, mn=256, seeds=1, cancellations=(1.0, 2.0 ** -12),
+                                            k_cancel=512, ks_coherent=(16, 512))
+    by = {r["case"]: r for r in rows}
+    for r in rows:
+        # truncating accumulation doubles the unit roundoff of the k additions (the test gate)
+        for m in ("termwise", "elementwise", "four_term"):
+            assert r[m + "_eta"] <= max(2 * r["k"], r["k"] + 14), (r["case"], m, r[m + "_eta"])
+    # cancellation leaves the componentwise error alone and ruins the relative error of entries
+    assert by["cancel c=2^-12"]["termwise_eta"] < 4 * by["cancel c=2^0"]["termwise_eta"] + 2
+    assert by["cancel c=2^-12"]["termwise_maxrel"] > 50 * by["cancel c=2^0"]["termwise_maxrel"]
+    # coherent residuals: the dropped term shows in full (about 2^-22 = 4 u_32 / 1.05^2), the
+    # four-term variant removes it
+    r = by["coherent residuals k=16"]
+    assert r["termwise_eta"] - r["four_term_eta"] > 2.0

@@ -126,3 +126,20 @@ def test_invalid_arguments():
     A = np.zeros((2, 3), np.float32)
     with pytest.raises(ValueError):
         oracle.sgemm_cube_four_term(A, np.zeros((4, 2), np.float32))
+
+
+def test_coherent_residuals_show_the_dropped_term_in_full():
+    # Constructed inputs: every entry 1.xx + (just under) half a unit in the 11th place, so every
+    # residual is about +2^-11 relative and the dropped products add up coherently:
+    # sum lo lo 2^-22 ~ 2^-22 / 1.05^2 of |A||B| = about 3.6 u_32, which the four-term sum recovers.
+    A = inputs.coherent_residuals(1, (32, 64), 0)
+    B = inputs.coherent_residuals(1, (64, 24), 1)
+    _, lo = oracle.split(A, 11)
+    assert np.all(lo.view(np.float16) > 0.99)
+    C64, ABabs = oracle.dgemm_ref(A, B)
+    e3 = (oracle.sgemm_cube(A, B, 11, oracle.TERMWISE, 64).astype(np.float64) - C64) / ABabs
+    e4 = (oracle.sgemm_cube_four_term(A, B, 11, 64).astype(np.float64) - C64) / ABabs
+    assert e3.mean() * 2.0 ** 24 < -3.0 and abs(e4.mean()) * 2.0 ** 24 < 0.5   # a bias, removed
+    shift = (e4 - e3).mean() * 2.0 ** 24
+    assert 3.0 < shift < 4.0
+    assert np.abs(e4).max() < np.abs(e3).max()

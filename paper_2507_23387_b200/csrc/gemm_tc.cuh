@@ -391,7 +391,6 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA0, const __grid_constant__
           SGC_TADD(13, blockIdx.x == 1 && threadIdx.x == 0);
         }
         SGC_T0();
-        if (with_x && !wait_tfull(1)) { ok = false; break; }
         tc_fence_after_sync();
         const uint32_t t_main = tmem_base + lane_addr + r_main * kBN + half * 128;
         const uint32_t t_x = tmem_base + lane_addr + kBN + half * 128;
@@ -407,24 +406,31 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA0, const __grid_constant__
 #pragma unroll
             for (int j = 0; j < GW; ++j) S[g * GW + j] = __fadd_rn(S[g * GW + j], __uint_as_float(v[j]));
           }
-          if (with_x) {
-            // Elementwise: fold this k-block's corrections into the same accumulator.
+        }
+        tc_fence_before_sync();
+        __syncwarp();
+        if (lane == 0) arrive_tempty(r_main);
+        drains[r_main]++;
+        if (with_x) {
+          // Elementwise: fold this k-block's corrections into the same accumulator, after its
+          // hi*hi sum (the bracketing of Eq. elementwise).  The hi*hi region has already gone back
+          // to the MMA thread, whose next hi*hi products run while this region is read.
+          if (!wait_tfull(1)) { ok = false; break; }
+          tc_fence_after_sync();
+#pragma unroll
+          for (int g = 0; g < 128 / GW; ++g) {
+            uint32_t v[GW];
             tmem_ld_cols(t_x + g * GW, v);
             tmem_ld_wait();
 #pragma unroll
             for (int j = 0; j < GW; ++j)
               S[g * GW + j] = __fadd_rn(S[g * GW + j], __fmul_rn(__uint_as_float(v[j]), p.inv_scale));
           }
+          tc_fence_before_sync();
+          __syncwarp();
+          if (lane == 0) arrive_tempty(1);
+          drains[1]++;
         }
-        tc_fence_before_sync();
-        __syncwarp();
-        SGC_TADD(15, blockIdx.x == 1 && threadIdx.x == 0);
-        if (lane == 0) {
-          arrive_tempty(r_main);
-          if (with_x) arrive_tempty(1);
-        }
-        drains[r_main]++;
-        if (with_x) drains[1]++;
         SGC_TADD(7, blockIdx.x == 0 && threadIdx.x == 0);
         SGC_TADD(14, blockIdx.x == 1 && threadIdx.x == 0);
       }
@@ -677,6 +683,21 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA0, const __grid_constant__
               continue;
             }
 #endif
+            if (NTERMS == 3 && p.order == 1) {
+              // Elementwise: both regions go to the accumulate warps after every k-block.  hi*hi
+              // first and handed over at once: it is drained while the correction products run,
+              // and the corrections are drained while the next block's hi*hi products run.
+              ok = stage_ready(it, st) && issue_main(st, it, first_kb, /*release*/ false);
+              if (!ok) break;
+              if (kb == kb_end - 1) {
+                commit_both(&tfull_bar[r_main]);
+                fills[r_main]++;
+                handed_over = true;
+              }
+              ok = issue_cross(st, first_kb);
+              commit_both(&empty_bar[it % STAGES]);
+              continue;
+            }
             ok = stage_ready(it, st) && (NTERMS != 3 || issue_cross(st, first_kb)) &&
                  issue_main(st, it, first_kb);
           }

@@ -287,7 +287,7 @@ int launch_tc_gemm(sgemm_cube_ctx* h, int M, int N, int K, const uint16_t* Ahi, 
   // Split-K: when the tiles would leave more than half of the SMs idle and k is long, cut the k
   // range into slices (whole k-blocks) so that tiles x slices fills the machine; a reduction
   // kernel adds the slices' sums.
-  bool pair = use_pair(h, M, N, false) && !Dll;
+  bool pair = use_pair(h, M, N, false);
   // Split-K runs on single CTAs; with the pair mode left to the library it takes precedence.
   if (NTERMS == 3 && h->split_k && (!pair || h->cta_pair == 2)) {
     const int tiles = ((M + sgc::kBM - 1) / sgc::kBM) * ((N + sgc::kBN - 1) / sgc::kBN);
@@ -323,7 +323,9 @@ int launch_tc_gemm(sgemm_cube_ctx* h, int M, int N, int K, const uint16_t* Ahi, 
     p.ldp = (long long)ldp;
   }
   if (p.Phh) {
-    rc = launch_tc_kernel<NTERMS, false, false>(h, M, N, tmA0, tmA1, tmB0, tmB1, p, st);
+    // raw sums to the workspace: k slices on single CTAs, or (four-term path, one slice) pairs
+    rc = (pair && p.ksplit == 1) ? launch_tc_kernel<NTERMS, false, true>(h, M, N, tmA0, tmA1, tmB0, tmB1, p, st)
+                                 : launch_tc_kernel<NTERMS, false, false>(h, M, N, tmA0, tmA1, tmB0, tmB1, p, st);
     if (rc) return rc;
     const long long total = (long long)M * N;
     long long blocks = (total + 255) / 256;

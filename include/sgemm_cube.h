@@ -153,6 +153,10 @@ int sgemm_cube_split(sgemm_cube_handle h, int rows, int cols,
  * problems are valid in every GEMM entry point of this header: M == 0 or N == 0 does nothing,
  * K == 0 stores C = 0 (the empty sum; left alone by sgemm_cube_hgemm with accumulate != 0); an
  * operand without elements may be a null pointer.
+ * Once the workspace for a problem size exists (after the first call at that size or a larger
+ * one) the call only enqueues work on `stream`: it can be captured into a CUDA graph and replayed.
+ * A handle's workspace is shared by its calls, so calls that may overlap on the GPU need one
+ * handle per stream.
  * Errors: INVALID_ARG, MISALIGNED, CUDA_ERROR (ALLOC_FAILED only with the TWO_PHASE strategy
  * forced; AUTO falls back to the fused kernel when the workspace cannot be had). */
 int sgemm_cube(sgemm_cube_handle h, int M, int N, int K,

@@ -355,6 +355,20 @@ def main():
         sm_max = clocks.get("sm_max_mhz") or 1965.0
         clock_peak = sm_count * 8192 * sm_max * 1e6 / 1e12       # dense FP16 flop/clk/SM x clock
         cpu_val, cpu_s, cpu_threads = cpu_oracle_sample(args.cpu_rows)
+        # Error of the step's result against an FP64 product, on 256 sampled rows (the second half
+        # of the metric: "max rel err vs FP64").  Componentwise: |C - C64| / (|A||B|), the quantity
+        # the method's bound (Eq. main_bound) and the test gate 2 K 2^-24 are stated in.
+        h.sgemm_cube(A, B, C, SCALE_EXP, binding.TERMWISE)
+        rows_idx = torch.arange(0, M, max(M // 256, 1), device=dev)[:256]
+        A64 = A[rows_idx].double()
+        C64 = A64 @ B.double()
+        AB = A64.abs() @ B.double().abs()
+        diff = (C[rows_idx].double() - C64).abs()
+        accuracy = {"rows_sampled": int(rows_idx.numel()),
+                    "frobenius_rel_err": float(diff.norm() / C64.norm()),
+                    "max_componentwise_err": float((diff / AB).max()),
+                    "componentwise_gate_2K_u32": 2.0 * K * 2.0 ** -24}
+        del A64, C64, AB, diff
         out = {
             "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
             "warmup": warmup, "ms_per_step": ms_per_step, "higher_is_better": True,
@@ -385,6 +399,7 @@ def main():
                              "sample": "%d of %d rows of A against the full B, %.1f s"
                                        % (args.cpu_rows, M, cpu_s)},
             "ablation": extra,
+            "accuracy": accuracy,
             "paper_context": "65.3 TFLOP/s = 77% of 256/3 on Ascend 910A (other hardware; not a target)",
         }
         print(json.dumps(out))

@@ -41,7 +41,7 @@ typedef struct sgemm_cube_ctx* sgemm_cube_handle;
 /* status codes */
 enum {
   SGEMM_CUBE_OK = 0,
-  SGEMM_CUBE_INVALID_ARG = 1,      /* null pointer, non-positive size, ld too small, bad enum   */
+  SGEMM_CUBE_INVALID_ARG = 1,      /* null pointer, negative size, ld too small, bad enum        */
   SGEMM_CUBE_MISALIGNED = 2,       /* pointer / leading dimension violates an alignment rule    */
   SGEMM_CUBE_CUDA_ERROR = 3,       /* a CUDA runtime or driver call failed                      */
   SGEMM_CUBE_DEVICE_TIMEOUT = 4,   /* a kernel gave up on a bounded wait (see sgemm_cube_check) */

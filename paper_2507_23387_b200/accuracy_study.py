@@ -183,6 +183,45 @@ def adversarial_sweep(h, mn=1024, seeds=3, scale_exp=11, device="cuda:0",
     return rows
 
 
+def config_errors(h, device="cuda:0", rows_sampled=512):
+    """Errors at the benchmark configurations (sizes and input distributions of the build's five
+    workloads), both accumulation orders, against an FP64 product on `rows_sampled` rows:
+    Frobenius relative error and the largest componentwise error in units of 2^-24."""
+    configs = [("256^3 U[-1,1)", "uniform_pm1", 256, 256, 256),
+               ("4096^3 U[-1,1)", "uniform_pm1", 4096, 4096, 4096),
+               ("8192^3 exponent spread", "exponent_spread", 8192, 8192, 8192),
+               ("1024 x 1024 x 65536 N(0,1)", "normal", 1024, 1024, 65536),
+               ("2048^3 N(0,1)", "normal", 2048, 2048, 2048),
+               ("16384 x 16384 x 1024 N(0,1)", "normal", 16384, 16384, 1024)]
+    rows = []
+    for name, kind, M, N, K in configs:
+        A_h, B_h = inputs.make_pair(kind, 0, M, N, K)
+        A, B = torch.from_numpy(A_h).to(device), torch.from_numpy(B_h).to(device)
+        del A_h, B_h
+        C = torch.empty((M, N), device=device)
+        idx = torch.arange(0, M, max(M // rows_sampled, 1), device=device)[:rows_sampled]
+        A64 = A[idx].double()
+        B64 = B.double()
+        C64 = A64 @ B64
+        AB = A64.abs() @ B64.abs()
+        del B64
+        r = {"config": name, "gate_2k": 2.0 * K}
+        for oname, order in (("termwise", binding.TERMWISE), ("elementwise", binding.ELEMENTWISE)):
+            h.sgemm_cube(A, B, C, 11, order)
+            d = (C[idx].double() - C64).abs()
+            r[oname + "_frob"] = float(d.norm() / C64.norm())
+            r[oname + "_eta_u32"] = float((d / AB).max()) * 2.0 ** 24
+        d = (_fp32_gemm(A, B)[idx].double() - C64).abs()
+        r["fp32_gemm_frob"] = float(d.norm() / C64.norm())
+        r["fp32_gemm_eta_u32"] = float((d / AB).max()) * 2.0 ** 24
+        rows.append(r)
+        del A, B, C, A64, C64, AB, d
+    status, detail = h.sgemm_cube_check()
+    if status != 0:
+        raise RuntimeError("device error %s" % hex(detail))
+    return rows
+
+
 def _table(rows, key, cols):
     lines = ["| %s | %s |" % (key, " | ".join(cols)), "|" + "---|" * (len(cols) + 1)]
     for r in rows:
@@ -196,8 +235,18 @@ def main():
     ap.add_argument("--seeds", type=int, default=5)
     ap.add_argument("--quick", action="store_true")
     ap.add_argument("--json", action="store_true")
+    ap.add_argument("--configs", action="store_true",
+                    help="only the error table at the benchmark configurations")
     args = ap.parse_args()
     h = binding.Handle(0)
+    if args.configs:
+        rows = config_errors(h)
+        h.destroy()
+        print("## Errors at the benchmark configurations (s_b = 11, default k-blocks), against FP64 on "
+              "512 sampled rows\n")
+        print(_table(rows, "config", ["gate_2k", "termwise_frob", "elementwise_frob", "fp32_gemm_frob",
+                                      "termwise_eta_u32", "elementwise_eta_u32", "fp32_gemm_eta_u32"]))
+        return
     exps = range(-12, 3, 4) if args.quick else range(-16, 5, 2)
     cols = ["fp16_hgemm", "fp32_gemm", "termwise_s0", "elementwise_s0", "termwise_s6", "termwise_s11",
             "termwise_s12", "elementwise_s12"]

@@ -317,6 +317,28 @@ def test_config5_large_shapes_sampled_rows(handle, shape):
     assert torch.equal(C2, C[:256][perm])
 
 
+@pytest.mark.parametrize("strategy", ["two_phase", "fused"])
+def test_operands_beyond_2_pow_31_elements(handle, strategy):
+    # A has 2.18e9 elements (8.7 GB): element offsets of its last rows, of the FP16 word matrices
+    # and of the workspace need 64 bits.  Rows from both ends are checked against the oracle.
+    M, N, K = 66000, 8, 33000
+    A = inputs.device_normal(3, (M, K))
+    B = inputs.device_normal(4, (K, N))
+    C = torch.full((M, N), float("nan"), device="cuda:0")
+    handle.sgemm_cube_set_option(binding.OPT_STRATEGY, STRATEGY[strategy])
+    try:
+        handle.sgemm_cube(A, B, C, 11, T)
+    finally:
+        handle.sgemm_cube_set_option(binding.OPT_STRATEGY, binding.STRATEGY_AUTO)
+    assert handle.sgemm_cube_check()[0] == 0
+    assert torch.isfinite(C).all()
+    rows = np.array([0, 1, 127, 128, 32768, 65071, 65072, 65535, 65998, 65999])
+    idx = torch.as_tensor(rows, device="cuda:0")
+    gates(C[idx].cpu().numpy(), A[idx].cpu().numpy(), B.cpu().numpy(), 11, T, label="2^31 " + strategy)
+    del A, B, C
+    torch.cuda.empty_cache()
+
+
 def test_hgemm_matches_fp64_product_of_fp16_inputs(handle):
     for (M, N, K) in [(128, 256, 64), (200, 300, 136), (1024, 1024, 1024)]:
         A = inputs.normal(1, (M, (K + 7) // 8 * 8))[:, :K]

@@ -339,6 +339,34 @@ def test_operands_beyond_2_pow_31_elements(handle, strategy):
     torch.cuda.empty_cache()
 
 
+def test_b_and_c_beyond_2_pow_31_elements(handle):
+    # B with 2.18e9 elements (columns of its last rows are far beyond 2^31), then C with 2.15e9.
+    K, N = 33000, 66000
+    A = inputs.device_normal(5, (8, K))
+    B = inputs.device_normal(6, (K, N))
+    C = torch.full((8, N), float("nan"), device="cuda:0")
+    handle.sgemm_cube(A, B, C, 11, T)
+    assert handle.sgemm_cube_check()[0] == 0 and torch.isfinite(C).all()
+    cols = np.array([0, 255, 256, 40000, 65535, 65999])
+    cidx = torch.as_tensor(cols, device="cuda:0")
+    gates(C[:, cidx].cpu().numpy(), A.cpu().numpy(), B[:, cidx].cpu().numpy(), 11, T, label="B > 2^31")
+    del A, B, C
+    torch.cuda.empty_cache()
+    M = N = 46400
+    A = inputs.device_normal(7, (M, 16))
+    B = inputs.device_normal(8, (16, N))
+    C = torch.full((M, N), float("nan"), device="cuda:0")
+    handle.sgemm_cube(A, B, C, 11, T)
+    assert handle.sgemm_cube_check()[0] == 0
+    rows = np.array([0, 127, 30000, 46271, 46272, 46399])
+    ridx = torch.as_tensor(rows, device="cuda:0")
+    Crows = C[ridx]
+    assert torch.isfinite(Crows).all() and torch.isfinite(C[:, N - 1]).all()
+    gates(Crows.cpu().numpy(), A[ridx].cpu().numpy(), B.cpu().numpy(), 11, T, label="C > 2^31")
+    del A, B, C
+    torch.cuda.empty_cache()
+
+
 def test_hgemm_matches_fp64_product_of_fp16_inputs(handle):
     for (M, N, K) in [(128, 256, 64), (200, 300, 136), (1024, 1024, 1024)]:
         A = inputs.normal(1, (M, (K + 7) // 8 * 8))[:, :K]

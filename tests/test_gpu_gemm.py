@@ -367,6 +367,31 @@ def test_b_and_c_beyond_2_pow_31_elements(handle):
     torch.cuda.empty_cache()
 
 
+@pytest.mark.parametrize("path,order", [("fused", T), ("fused", E), ("two_phase", T), ("two_phase", E)])
+def test_special_values_propagate_like_the_oracle(handle, path, order):
+    # inf, NaN, values beyond the FP16 range (hi = inf), zero rows and columns: IEEE semantics end
+    # to end (nothing is clamped), so every entry has the class (NaN / +inf / -inf / finite) the
+    # oracle gives it, and the rows and columns that saw no special value pass the usual gates.
+    A, B = inputs.make_pair("uniform_pm1", 1, 130, 260, 96)
+    A, B = A.copy(), B.copy()
+    A[3, 5], A[7, 9], A[11, 2], A[20, 0], A[21, 1] = np.inf, -np.inf, np.nan, 70000.0, -1e30
+    B[4, 17], B[50, 100] = np.inf, np.nan
+    A[40, :] = 0
+    B[:, 200] = 0
+    C = run(handle, path, to_dev(A), to_dev(B), 11, order)
+    Co = oracle.sgemm_cube(A, B, 11, order, K_BLOCK[order])
+
+    def cls(x):
+        return np.where(np.isnan(x), 2, np.where(np.isinf(x), np.sign(x), 0)).astype(np.int8)
+    assert np.array_equal(cls(C), cls(Co))
+    assert np.all(C[40, np.isfinite(C[40])] == 0) and np.all(C[np.isfinite(C[:, 200]), 200] == 0)
+    clean_rows = [i for i in range(130) if i not in (3, 7, 11, 20, 21)]
+    clean_cols = [j for j in range(260) if j not in (17, 100)]
+    sub = C[np.ix_(clean_rows, clean_cols)]
+    gates(sub, np.ascontiguousarray(A[clean_rows]), np.ascontiguousarray(B[:, clean_cols]), 11, order,
+          label="rows and columns without special values")
+
+
 def test_hgemm_matches_fp64_product_of_fp16_inputs(handle):
     for (M, N, K) in [(128, 256, 64), (200, 300, 136), (1024, 1024, 1024)]:
         A = inputs.normal(1, (M, (K + 7) // 8 * 8))[:, :K]

@@ -72,3 +72,25 @@ def test_input_scaling_choice_is_host_arithmetic(lib):
     for ra, rb in [([-14, 15, 0], [-14, 15, 0]), ([-40, -20, 0], [3, 20, 0]), ([0, 0, 1], [0, 0, 0]),
                    ([127, -127, 0], [5, 9, 0])]:
         assert binding.sgemm_cube_choose_input_scaling(ra, rb) == oracle.input_scale_exps(ra, rb)
+
+
+def test_binding_constants_match_the_header():
+    text = open(os.path.join(ROOT, "include", "sgemm_cube.h")).read()
+    text = re.sub(r"/\*.*?\*/", "", text, flags=re.S)
+    values = {m.group(1): int(m.group(2)) for m in re.finditer(r"\b(SGEMM_CUBE_\w+)\s*=\s*(\d+)", text)}
+    pairs = {"SGEMM_CUBE_OK": binding.OK, "SGEMM_CUBE_INVALID_ARG": binding.INVALID_ARG,
+             "SGEMM_CUBE_MISALIGNED": binding.MISALIGNED, "SGEMM_CUBE_CUDA_ERROR": binding.CUDA_ERROR,
+             "SGEMM_CUBE_DEVICE_TIMEOUT": binding.DEVICE_TIMEOUT,
+             "SGEMM_CUBE_UNSUPPORTED_ARCH": binding.UNSUPPORTED_ARCH,
+             "SGEMM_CUBE_ALLOC_FAILED": binding.ALLOC_FAILED, "SGEMM_CUBE_TOO_LARGE": binding.TOO_LARGE,
+             "SGEMM_CUBE_TERMWISE": binding.TERMWISE, "SGEMM_CUBE_ELEMENTWISE": binding.ELEMENTWISE,
+             "SGEMM_CUBE_OPT_TERMWISE_K_BLOCK": binding.OPT_TERMWISE_K_BLOCK,
+             "SGEMM_CUBE_OPT_ELEMENTWISE_K_BLOCK": binding.OPT_ELEMENTWISE_K_BLOCK,
+             "SGEMM_CUBE_OPT_CTA_PAIR": binding.OPT_CTA_PAIR, "SGEMM_CUBE_OPT_STRATEGY": binding.OPT_STRATEGY,
+             "SGEMM_CUBE_OPT_TIME_KERNEL": binding.OPT_TIME_KERNEL, "SGEMM_CUBE_OPT_SPLIT_K": binding.OPT_SPLIT_K,
+             "SGEMM_CUBE_STRATEGY_AUTO": binding.STRATEGY_AUTO, "SGEMM_CUBE_STRATEGY_FUSED": binding.STRATEGY_FUSED,
+             "SGEMM_CUBE_STRATEGY_TWO_PHASE": binding.STRATEGY_TWO_PHASE}
+    for name, val in pairs.items():
+        assert values.get(name) == val, name
+    m = re.search(r"SGEMM_CUBE_STATIC_SCRATCH_BYTES\s*\((\d+)u\s*<<\s*(\d+)\)", text)
+    assert m and int(m.group(1)) << int(m.group(2)) == binding.STATIC_SCRATCH_BYTES

@@ -250,6 +250,19 @@ int sgemm_cube_exponent_window(sgemm_cube_handle h, int rows, int cols,
                                const float* X_dev, int64_t ldx,
                                int64_t* window_out, void* stream);
 
+/* Residual-overflow detection (paper Sec. 4.2, Rule 2: "... unless residual overflow is explicitly
+ * detected and handled"): the number of entries of a split operand whose high word is finite
+ * while its scaled residual word is inf or NaN, i.e. for which (x - hi) 2^s left the FP16 range
+ * (the paper's example: x = 32784 at s_b = 12).  A non-zero count means the chosen scale exponent
+ * is too large for this operand; sgemm_cube_choose_scale_exp gives one that cannot overflow.
+ * One pass over the two word matrices; the call synchronises `stream`.
+ *   hi_dev, lo_dev  rows x cols FP16 bit patterns as written by sgemm_cube_split, ldh >= cols
+ *   count_out       1 x int64 (host, written)
+ * Errors: INVALID_ARG, CUDA_ERROR. */
+int sgemm_cube_residual_overflow_count(sgemm_cube_handle h, int rows, int cols,
+                                       const uint16_t* hi_dev, const uint16_t* lo_dev, int64_t ldh,
+                                       int64_t* count_out, void* stream);
+
 /* Scale exponent for a pair of operands from their exponent windows (host arithmetic only).
  * Eq. sf_bounds:  -3 - e_min <= s_b <= 26 - e_max  over both operands; following Sec. 4.2 ("scale
  * the residual as far from the underflow threshold as the largest entry permits") the upper end

@@ -251,3 +251,12 @@ def sgemm_cube_scaled(A, B, p_a, p_b, s=11, order=TERMWISE, kb=64):
     B2 = np.ldexp(np.asarray(B, dtype=np.float32), int(p_b)).astype(np.float32)
     C = sgemm_cube(A2, B2, s=s, order=order, kb=kb)
     return np.ldexp(C, -(int(p_a) + int(p_b))).astype(np.float32)
+
+
+def residual_overflow_count(X, s):
+    """Number of entries whose high word is finite while the scaled residual word is inf or NaN
+    (Rule 2 of Sec. 4.2 violated for that entry): counted on the words of the pinned split."""
+    hi, lo = split(np.atleast_2d(np.asarray(X, dtype=np.float32)), s)
+    hi_finite = (hi & 0x7C00) != 0x7C00
+    lo_nonfinite = (lo & 0x7C00) == 0x7C00
+    return int((hi_finite & lo_nonfinite).sum())

@@ -23,7 +23,7 @@ EXPORTS = ["sgemm_cube_create", "sgemm_cube_destroy", "sgemm_cube_set_option", "
            "sgemm_cube_four_term", "sgemm_cube_hi_exponent_range", "sgemm_cube_choose_input_scaling",
            "sgemm_cube_scaled", "sgemm_cube_auto_scaled",
            "sgemm_cube_host", "sgemm_cube_unfused_static", "sgemm_cube_check", "sgemm_cube_launch_count", "sgemm_cube_last_kernel_ms", "sgemm_cube_mean_kernel_ms",
-           "sgemm_cube_exponent_window", "sgemm_cube_choose_scale_exp",
+           "sgemm_cube_exponent_window", "sgemm_cube_choose_scale_exp", "sgemm_cube_residual_overflow_count",
            "sgemm_cube_status_string", "sgemm_cube_version"]
 
 _lib = None
@@ -67,6 +67,7 @@ def load():
     lib.sgemm_cube_last_kernel_ms.argtypes = [vp, ctypes.POINTER(ctypes.c_float)]
     lib.sgemm_cube_mean_kernel_ms.argtypes = [vp, ctypes.POINTER(ctypes.c_float), ctypes.POINTER(i32)]
     lib.sgemm_cube_exponent_window.argtypes = [vp, i32, i32, vp, i64, ctypes.POINTER(i64), vp]
+    lib.sgemm_cube_residual_overflow_count.argtypes = [vp, i32, i32, vp, vp, i64, ctypes.POINTER(i64), vp]
     lib.sgemm_cube_choose_scale_exp.argtypes = [ctypes.POINTER(i64), ctypes.POINTER(i64),
                                                 ctypes.POINTER(i32), ctypes.POINTER(i32)]
     lib.sgemm_cube_launch_count.argtypes = [vp]
@@ -199,6 +200,17 @@ class Handle:
                                            _dev(B, torch.float32), _ld(B), _dev(C, torch.float32),
                                            _ld(C), scale_exp, _stream_ptr(stream)),
                "sgemm_cube_four_term")
+
+    def sgemm_cube_residual_overflow_count(self, hi, lo, stream=None):
+        """Entries whose high word is finite while the scaled residual word is not."""
+        rows, cols = hi.shape
+        assert lo.shape == hi.shape and _ld(hi) == _ld(lo)
+        out = ctypes.c_int64(0)
+        _check(load().sgemm_cube_residual_overflow_count(self._h, rows, cols, _dev(hi, torch.float16),
+                                                         _dev(lo, torch.float16), _ld(hi),
+                                                         ctypes.byref(out), _stream_ptr(stream)),
+               "sgemm_cube_residual_overflow_count")
+        return int(out.value)
 
     def sgemm_cube_hi_exponent_range(self, X, stream=None):
         """[e_min, e_max, #inf/NaN] of the unbounded-range high-word exponents of X."""

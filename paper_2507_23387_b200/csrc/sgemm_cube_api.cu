@@ -963,6 +963,38 @@ int sgemm_cube_auto_scaled(sgemm_cube_handle h, int M, int N, int K, const float
   return sgemm_cube_scaled(h, M, N, K, A, lda, B, ldb, C, ldc, p_a, p_b, s, order, stream);
 }
 
+int sgemm_cube_residual_overflow_count(sgemm_cube_handle h, int rows, int cols, const uint16_t* hi,
+                                       const uint16_t* lo, int64_t ldh, int64_t* count_out, void* stream) {
+  if (!h || !count_out) return SGEMM_CUBE_INVALID_ARG;
+  if (rows < 0 || cols < 0 || ldh < cols) return SGEMM_CUBE_INVALID_ARG;
+  *count_out = 0;
+  if (rows == 0 || cols == 0) return SGEMM_CUBE_OK;
+  if (!hi || !lo) return SGEMM_CUBE_INVALID_ARG;
+  DeviceGuard g(h->device);
+  if (!g.ok) return SGEMM_CUBE_CUDA_ERROR;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  unsigned long long* dev = reinterpret_cast<unsigned long long*>(h->err_dev + 4);
+  if (cudaMemsetAsync(dev, 0, sizeof(unsigned long long), st) != cudaSuccess) {
+    cudaGetLastError();
+    return SGEMM_CUBE_CUDA_ERROR;
+  }
+  const long long total = (long long)rows * cols;
+  long long blocks = (total + 1023) / 1024;
+  const long long cap = (long long)h->sm_count * 16;
+  if (blocks > cap) blocks = cap;
+  sgc::residual_overflow_kernel<<<(unsigned)blocks, 256, 0, st>>>(rows, cols, hi, lo, ldh, dev);
+  h->launches++;
+  if (cudaGetLastError() != cudaSuccess) return SGEMM_CUBE_CUDA_ERROR;
+  unsigned long long res = 0;
+  if (cudaMemcpyAsync(&res, dev, sizeof(res), cudaMemcpyDeviceToHost, st) != cudaSuccess ||
+      cudaStreamSynchronize(st) != cudaSuccess) {
+    cudaGetLastError();
+    return SGEMM_CUBE_CUDA_ERROR;
+  }
+  *count_out = (int64_t)res;
+  return SGEMM_CUBE_OK;
+}
+
 int sgemm_cube_choose_scale_exp(const int64_t* window_a, const int64_t* window_b, int* scale_exp_out,
                                 int* protected_out) {
   if (!window_a || !window_b || !scale_exp_out) return SGEMM_CUBE_INVALID_ARG;

@@ -243,6 +243,26 @@ scale_pow2_kernel(int rows, int cols, float* __restrict__ C, long long ldc, int 
   }
 }
 
+// Residual-overflow detection (the "explicitly detected" alternative of Rule 2, Sec. 4.2): counts
+// the entries whose high word is finite while the scaled residual is not, i.e. entries for which
+// (x - hi) * 2^s left the FP16 range (the worked example of Sec. 4.2: x = 32784, s = 12).
+// out[0] += count.  HBM-bound: 4 bytes read per element.
+__global__ void __launch_bounds__(256)
+residual_overflow_kernel(int rows, int cols, const uint16_t* __restrict__ hi,
+                         const uint16_t* __restrict__ lo, long long ldh, unsigned long long* out) {
+  unsigned int n = 0;
+  const long long total = (long long)rows * cols;
+  const long long stride = (long long)gridDim.x * blockDim.x;
+  for (long long it = (long long)blockIdx.x * blockDim.x + threadIdx.x; it < total; it += stride) {
+    const long long r = it / cols;
+    const long long c = it - r * cols;
+    const unsigned int h = hi[r * ldh + c], l = lo[r * ldh + c];
+    if ((h & 0x7C00u) != 0x7C00u && (l & 0x7C00u) == 0x7C00u) ++n;
+  }
+  for (int o = 16; o > 0; o >>= 1) n += __shfl_xor_sync(0xffffffffu, n, o);
+  if ((threadIdx.x & 31) == 0 && n) atomicAdd(out, (unsigned long long)n);
+}
+
 // Split-K reduction: C = sum_s Phh[s] + inv_scale * sum_s Px[s] (termwise: the slices' hi*hi sums
 // and correction sums are added among themselves, in slice order, and meet once), or
 // C = sum_s Phh[s] (elementwise: each slice's running accumulator).  FP32 RN additions.

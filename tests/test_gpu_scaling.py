@@ -58,3 +58,19 @@ def test_chosen_scale_keeps_the_split_inside_its_error_bound(handle):
     rec = hi.double().cpu().numpy() + lo.double().cpu().numpy() * 2.0 ** -s
     assert np.isfinite(rec).all()
     assert np.all(np.abs(rec - X.astype(np.float64)) <= 2.0 ** -22 * np.abs(X.astype(np.float64)))
+
+
+def test_residual_overflow_count_matches_oracle(handle):
+    V = np.array([[32784.0, 1.0, -32784.0, 0.5, 70000.0, np.inf, np.nan, 65000.0]], dtype=np.float32)
+    X = inputs.exponent_spread(9, (300, 520), 5, 15)
+    for src in (V, X):
+        for s in (0, 8, 11, 12, 15):
+            Xd = to_dev(src)
+            hi = torch.empty(Xd.shape, dtype=torch.float16, device="cuda:0")
+            lo = torch.empty_like(hi)
+            handle.sgemm_cube_split(Xd, hi, lo, s)
+            assert handle.sgemm_cube_residual_overflow_count(hi, lo) == oracle.residual_overflow_count(src, s)
+    # what sgemm_cube_choose_scale_exp returns never overflows a residual
+    win = handle.sgemm_cube_exponent_window(to_dev(X))
+    s, _ = binding.sgemm_cube_choose_scale_exp(win, win)
+    assert oracle.residual_overflow_count(X, s) == 0 and oracle.residual_overflow_count(X, 15) > 0

@@ -115,3 +115,19 @@ def test_scaling_restores_the_accuracy_of_tiny_inputs():
     assert pa == 15 - ra[1] and pa >= 44
     scaled = oracle.frobenius_rel_err(oracle.sgemm_cube_scaled(A, B, pa, pb, s, oracle.TERMWISE, 64), C64)
     assert plain > 0.5 and scaled < 5e-7
+
+
+def test_residual_overflow_detection_on_the_papers_example():
+    # Sec. 4.2: V = 32784 rounds to 32768, residual 16; 16 * 2^12 = 65536 overflows FP16, 16 * 2^11
+    # does not.  Rule 2: s_b <= 26 - e_max with e_max = 15 here.
+    V = np.array([[32784.0, 1.0, -32784.0, 0.5]], dtype=np.float32)
+    assert oracle.residual_overflow_count(V, 12) == 2
+    assert oracle.residual_overflow_count(V, 11) == 0
+    # inputs beyond the FP16 range (hi = inf) are not residual overflows
+    assert oracle.residual_overflow_count(np.array([[70000.0, np.inf, np.nan]], dtype=np.float32), 12) == 0
+    # the bound of Rule 2 is exactly where overflow can start: ties at exponent e overflow at 27 - e
+    for e in range(3, 16):
+        x = np.array([[2.0 ** e * (1 + 2.0 ** -11)]], dtype=np.float32)
+        assert oracle.residual_overflow_count(x, min(26 - e, 24)) == 0
+        if 27 - e <= 24:
+            assert oracle.residual_overflow_count(x, 27 - e) == 1

@@ -24,6 +24,7 @@ from .bounds import (U16, U32, gamma, tau, ll_coeff, main_bound_coeff,  # noqa: 
 
 TERMWISE = 0
 ELEMENTWISE = 1
+ELEMENTWISE_REORDERED = 2      # Sec. 4.5, last paragraph: corrections of a k-block summed first
 
 _lib = None
 

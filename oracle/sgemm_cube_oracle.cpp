@@ -13,6 +13,7 @@
 //     in a fixed order, k cut into blocks of kb:
 //        termwise     [Eq. termwise]     three streams, combined once at the end
 //        elementwise  [Eq. elementwise]  the three block products folded into one accumulator
+//        reordered elementwise [Sec. 4.5, last paragraph]  corrections of a block summed first
 //   * references: FP64 GEMM, |A||B| in FP64, sequential FP32 GEMM of the unsplit inputs,
 //     and the hi*hi product alone ("native FP16 GEMM" contrast)    [Sec. 6.1, 6.2]
 //
@@ -132,7 +133,10 @@ void oracle_split(int64_t rows, int64_t cols, const float* X, int64_t ldx,
 }
 
 // C = hi_A hi_B + 2^-s (lo_A hi_B + hi_A lo_B), FP32 accumulation.   [Eq. recover_eqn]
-//   order 0: termwise [Eq. termwise]; order 1: elementwise [Eq. elementwise].
+//   order 0: termwise [Eq. termwise]; order 1: elementwise [Eq. elementwise]; order 2: the
+//   reordered elementwise variant of Sec. 4.5 (last paragraph): per k-block the two corrections
+//   are summed first, scaled, added to the block's hi*hi product, and the result is added to the
+//   accumulator once:  acc = acc + ((R_A^[g]B^[g] + A^[g]R_B^[g]) / s_f + A^[g]B^[g]).
 //   kb: size of a k-block g (one product A^[g] B^[g] is summed from zero over ascending k,
 //       every addition an FP32 RN addition; FP16 x FP16 products are exact in FP32 [Sec. 4.4]).
 //   Chgemm (optional): the hi*hi stream alone, summed the termwise way.
@@ -141,7 +145,7 @@ int oracle_sgemm_cube(int64_t M, int64_t N, int64_t K,
                       const float* A, int64_t lda, const float* B, int64_t ldb,
                       float* C, int64_t ldc, int s, int order, int64_t kb, float* Chgemm,
                       int64_t ldch) {
-  if (M < 0 || N < 0 || K < 0 || kb <= 0 || s < 0 || s > 24 || (order != 0 && order != 1))
+  if (M < 0 || N < 0 || K < 0 || kb <= 0 || s < 0 || s > 24 || order < 0 || order > 2)
     return 1;
   // Split B once; keep the FP16 words widened (exactly) to FP32 for the loops.
   std::vector<float> Bh((size_t)K * N), Bl((size_t)K * N);
@@ -187,7 +191,7 @@ int oracle_sgemm_cube(int64_t M, int64_t N, int64_t K,
             Slh[j] = Slh[j] + Plh[j];
             Shl[j] = Shl[j] + Phl[j];
           }
-        } else {
+        } else if (order == 1) {
           // ((acc + A^[g]B^[g]) + R_A^[g]B^[g]/s_f) + A^[g]R_B^[g]/s_f
           for (int64_t j = 0; j < N; ++j) {
             float acc = Shh[j];
@@ -195,6 +199,14 @@ int oracle_sgemm_cube(int64_t M, int64_t N, int64_t K,
             acc = acc + Plh[j] * inv_sf;
             acc = acc + Phl[j] * inv_sf;
             Shh[j] = acc;
+            Slh[j] = Slh[j] + Phh[j];          // hi*hi stream alone, for Chgemm
+          }
+        } else {
+          // acc + ((R_A^[g]B^[g] + A^[g]R_B^[g]) / s_f + A^[g]B^[g])
+          for (int64_t j = 0; j < N; ++j) {
+            const float cross = Plh[j] + Phl[j];
+            const float block = cross * inv_sf + Phh[j];
+            Shh[j] = Shh[j] + block;
             Slh[j] = Slh[j] + Phh[j];          // hi*hi stream alone, for Chgemm
           }
         }

@@ -67,6 +67,9 @@ def _brute_force(A, B, s, order, kb):
                     P[2] = _rn32(P[2] + Ah[i, k] * Bl[k, j])
                 if order == oracle.TERMWISE:
                     S = [_rn32(S[t] + P[t]) for t in range(3)]
+                elif order == oracle.ELEMENTWISE_REORDERED:
+                    block = _rn32(_rn32(P[1] + P[2]) * inv + P[0])
+                    acc = _rn32(acc + block)
                 else:
                     acc = _rn32(acc + P[0])
                     acc = _rn32(acc + P[1] * inv)
@@ -91,7 +94,7 @@ def test_rn32_helper_agrees_with_numpy_float32():
     assert _rn32(Fraction(2 ** 24 + 3)) == 2 ** 24 + 4
 
 
-@pytest.mark.parametrize("order", [oracle.TERMWISE, oracle.ELEMENTWISE])
+@pytest.mark.parametrize("order", [oracle.TERMWISE, oracle.ELEMENTWISE, oracle.ELEMENTWISE_REORDERED])
 @pytest.mark.parametrize("kb", [1, 3, 64])
 def test_small_integers_give_the_exact_product(order, kb):
     # Integers of magnitude <= 8: hi = x, lo = 0, every partial sum exact.  Non-square shapes and
@@ -105,7 +108,7 @@ def test_small_integers_give_the_exact_product(order, kb):
     assert np.array_equal(C.astype(np.int64), want) and np.array_equal(C, want.astype(np.float32))
 
 
-@pytest.mark.parametrize("order", [oracle.TERMWISE, oracle.ELEMENTWISE])
+@pytest.mark.parametrize("order", [oracle.TERMWISE, oracle.ELEMENTWISE, oracle.ELEMENTWISE_REORDERED])
 @pytest.mark.parametrize("s", [9, 11, 12])
 def test_three_terms_kept_and_low_low_dropped_exactly(order, s):
     # x = p + q 2^-13 with p in {4..7}, q in {-3..3}: hi = p, residual q 2^-13 exactly, and all
@@ -130,7 +133,7 @@ def test_three_terms_kept_and_low_low_dropped_exactly(order, s):
     assert np.allclose(full - C, dropped, rtol=0, atol=1e-15) and np.any(dropped != 0)
 
 
-@pytest.mark.parametrize("order", [oracle.TERMWISE, oracle.ELEMENTWISE])
+@pytest.mark.parametrize("order", [oracle.TERMWISE, oracle.ELEMENTWISE, oracle.ELEMENTWISE_REORDERED])
 @pytest.mark.parametrize("kb", [3, 7, 100])
 def test_brute_force_rounding_order_on_tiny_inputs(order, kb):
     M, N, K = 3, 2, 7
@@ -159,6 +162,26 @@ def test_orders_differ_matches_brute_force():
     tw = oracle.sgemm_cube(A, B, s=s, order=oracle.TERMWISE, kb=1)
     assert float(el[0, 0]) == 1 + 3 * 2.0 ** -12
     assert float(tw[0, 0]) == 1 + 3 * 2.0 ** -12 + 2.0 ** -23
+
+
+def test_reordered_elementwise_keeps_what_the_plain_order_loses_inside_a_block():
+    # Sec. 4.5, last paragraph: summing the two corrections of a block before they meet the large
+    # accumulator removes the swamping inside a block.  Block 0 makes the accumulator 1; block 1
+    # has hi*hi = 2^-12 and two corrections of 0.375 ulp(1) each: added one by one to 1 + 2^-12
+    # both are lost, added together (0.75 ulp) they round up.
+    u = 2.0 ** -23
+    a = 2.0 ** -12 * (1 + 3 * 2.0 ** -14)          # hi = 2^-12, residual 3 * 2^-26
+    b = 1 + 3 * 2.0 ** -14                          # hi = 1,     residual 3 * 2^-14
+    A = np.array([[1.0, a]], dtype=np.float32)
+    B = np.array([[1.0], [b]], dtype=np.float32)
+    el = float(oracle.sgemm_cube(A, B, s=11, order=oracle.ELEMENTWISE, kb=1)[0, 0])
+    ro = float(oracle.sgemm_cube(A, B, s=11, order=oracle.ELEMENTWISE_REORDERED, kb=1)[0, 0])
+    tw = float(oracle.sgemm_cube(A, B, s=11, order=oracle.TERMWISE, kb=1)[0, 0])
+    assert el == 1 + 2.0 ** -12
+    assert ro == 1 + 2.0 ** -12 + u and tw == ro
+    for order in (oracle.ELEMENTWISE, oracle.ELEMENTWISE_REORDERED):
+        got = _to_frac_matrix(oracle.sgemm_cube(A, B, s=11, order=order, kb=1))
+        assert np.array_equal(got, _brute_force(A, B, 11, order, 1))
 
 
 @pytest.mark.parametrize("kind", ["uniform_pm1", "exponent_spread", "normal"])

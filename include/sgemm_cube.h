@@ -53,7 +53,12 @@ enum {
 /* accumulation order (paper Sec. 4.5) */
 enum {
   SGEMM_CUBE_TERMWISE = 0,   /* Eq. termwise: streams summed separately, combined once at the end */
-  SGEMM_CUBE_ELEMENTWISE = 1 /* Eq. elementwise: per k-block, products folded into one accumulator */
+  SGEMM_CUBE_ELEMENTWISE = 1, /* Eq. elementwise: per k-block, products folded into one accumulator */
+  /* The reordered elementwise order that Sec. 4.5 (last paragraph) proposes and leaves unmeasured:
+   * per k-block the corrections are summed first, scaled, added to the block's hi*hi product, and
+   * the block enters the accumulator once: acc = acc + ((R_A B + A R_B) / s_f + A B).  Uses the
+   * elementwise k-block option.  Accepted wherever an accumulation order is. */
+  SGEMM_CUBE_ELEMENTWISE_REORDERED = 2
 };
 
 /* options for sgemm_cube_set_option */
@@ -147,7 +152,8 @@ int sgemm_cube_split(sgemm_cube_handle h, int rows, int cols,
  *   A_dev  M x K FP32, lda >= K     (device, read)
  *   B_dev  K x N FP32, ldb >= N     (device, read)
  *   C_dev  M x N FP32, ldc >= N     (device, written)
- *   scale_exp s in [0, 24]; accumulation_order SGEMM_CUBE_TERMWISE or SGEMM_CUBE_ELEMENTWISE
+ *   scale_exp s in [0, 24]; accumulation_order SGEMM_CUBE_TERMWISE, SGEMM_CUBE_ELEMENTWISE or
+ *   SGEMM_CUBE_ELEMENTWISE_REORDERED
  * Alignment: A_dev, B_dev 16-byte aligned and lda % 4 == 0, ldb % 4 == 0 (else MISALIGNED).
  * C_dev may have any alignment.  M, N, K >= 0, any values (ragged edges are handled).  Empty
  * problems are valid in every GEMM entry point of this header: M == 0 or N == 0 does nothing,

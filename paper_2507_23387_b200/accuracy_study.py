@@ -5,7 +5,7 @@ Eq. err, mean over seeds):
 
   exponent sweep   entries U[-2^e, 2^e] (symmetric) or U[0, 2^e] (non-negative) for a range of
                    offset exponents e, scale exponents s_b in {0, 6, 11, 12}; compared methods:
-                   termwise and elementwise SGEMM-cube, the hi*hi product alone ("FP16 HGEMM"),
+                   termwise, elementwise and reordered-elementwise SGEMM-cube, the hi*hi product alone ("FP16 HGEMM"),
                    and an FP32 GEMM                                  (Fig. scaling_bit_error)
   size sweep       error against m = n, against k, and against all three, at offset exponent 0
                                                                       (Fig. mkn_error)
@@ -71,7 +71,8 @@ def measure(h, A, B, scale_exps=(0, 6, 11, 12)):
            "fp16_hgemm": frobenius_rel_err(_hgemm_hi_only(h, A, B, 0), C64)}
     C = torch.empty((M, N), device=A.device)
     for s in scale_exps:
-        for name, order in (("termwise", binding.TERMWISE), ("elementwise", binding.ELEMENTWISE)):
+        for name, order in (("termwise", binding.TERMWISE), ("elementwise", binding.ELEMENTWISE),
+                            ("reordered", binding.ELEMENTWISE_REORDERED)):
             h.sgemm_cube(A, B, C, s, order)
             out["%s_s%d" % (name, s)] = frobenius_rel_err(C, C64)
         h.sgemm_cube_four_term(A, B, C, s)
@@ -206,7 +207,8 @@ def config_errors(h, device="cuda:0", rows_sampled=512):
         AB = A64.abs() @ B64.abs()
         del B64
         r = {"config": name, "gate_2k": 2.0 * K}
-        for oname, order in (("termwise", binding.TERMWISE), ("elementwise", binding.ELEMENTWISE)):
+        for oname, order in (("termwise", binding.TERMWISE), ("elementwise", binding.ELEMENTWISE),
+                             ("reordered", binding.ELEMENTWISE_REORDERED)):
             h.sgemm_cube(A, B, C, 11, order)
             d = (C[idx].double() - C64).abs()
             r[oname + "_frob"] = float(d.norm() / C64.norm())
@@ -244,19 +246,20 @@ def main():
         h.destroy()
         print("## Errors at the benchmark configurations (s_b = 11, default k-blocks), against FP64 on "
               "512 sampled rows\n")
-        print(_table(rows, "config", ["gate_2k", "termwise_frob", "elementwise_frob", "fp32_gemm_frob",
-                                      "termwise_eta_u32", "elementwise_eta_u32", "fp32_gemm_eta_u32"]))
+        print(_table(rows, "config", ["gate_2k", "termwise_frob", "elementwise_frob", "reordered_frob",
+                                      "fp32_gemm_frob", "termwise_eta_u32", "elementwise_eta_u32",
+                                      "reordered_eta_u32", "fp32_gemm_eta_u32"]))
         return
     exps = range(-12, 3, 4) if args.quick else range(-16, 5, 2)
     cols = ["fp16_hgemm", "fp32_gemm", "termwise_s0", "elementwise_s0", "termwise_s6", "termwise_s11",
-            "termwise_s12", "elementwise_s12"]
+            "termwise_s12", "elementwise_s12", "reordered_s12"]
     sym = exponent_sweep(h, args.size, exps, args.seeds, nonneg=False)
     pos = exponent_sweep(h, args.size, exps, args.seeds, nonneg=True)
     k_fixed = 64 * 44
     mn = [(n, n, k_fixed) for n in ((512, 2048) if args.quick else (256, 1024, 4096))]
     ks = [(1024, 1024, k) for k in ((256, 4096) if args.quick else (256, 1024, 4096, 16384, 65536))]
     alls = [(n, n, n) for n in ((512, 2048) if args.quick else (512, 1024, 2048, 4096))]
-    scol = ["fp16_hgemm", "fp32_gemm", "termwise_s12", "elementwise_s12"]
+    scol = ["fp16_hgemm", "fp32_gemm", "termwise_s12", "elementwise_s12", "reordered_s12"]
     res = {"symmetric": sym, "nonnegative": pos, "vs_mn": size_sweep(h, mn, args.seeds),
            "vs_k": size_sweep(h, ks, args.seeds), "vs_all": size_sweep(h, alls, args.seeds),
            "dropped_term": dropped_term_sweep(h, (8, 512) if args.quick else (8, 32, 128, 512, 2048, 8192),

@@ -14,7 +14,7 @@ LIB_PATH = os.path.join(HERE, "libsgemm_cube.so")
 
 OK, INVALID_ARG, MISALIGNED, CUDA_ERROR, DEVICE_TIMEOUT, UNSUPPORTED_ARCH, ALLOC_FAILED, TOO_LARGE = range(8)
 STATIC_SCRATCH_BYTES = 32 << 20
-TERMWISE, ELEMENTWISE = 0, 1
+TERMWISE, ELEMENTWISE, ELEMENTWISE_REORDERED = 0, 1, 2
 OPT_TERMWISE_K_BLOCK, OPT_ELEMENTWISE_K_BLOCK, OPT_CTA_PAIR, OPT_STRATEGY, OPT_TIME_KERNEL, OPT_SPLIT_K = range(6)
 STRATEGY_AUTO, STRATEGY_FUSED, STRATEGY_TWO_PHASE = 0, 1, 2
 

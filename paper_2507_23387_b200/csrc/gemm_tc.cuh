@@ -256,7 +256,10 @@ __device__ __forceinline__ void tmem_ld_cols(uint32_t taddr, uint32_t (&r)[16]) 
 __device__ __forceinline__ void tmem_ld_cols(uint32_t taddr, uint32_t (&r)[32]) { tmem_ld_32x32b_x32(taddr, r); }
 __device__ __forceinline__ void tmem_ld_cols(uint32_t taddr, uint32_t (&r)[64]) { tmem_ld_32x32b_x64(taddr, r); }
 
-template <int NTERMS, bool FUSED, bool PAIR>
+// REORD: the reordered elementwise order (p.order == 2) has its own instantiations, so that its
+// accumulate path (two chunk buffers live at once) does not weigh on the register allocation of
+// the termwise / elementwise kernels.
+template <int NTERMS, bool FUSED, bool PAIR, bool REORD = false>
 __global__ void __launch_bounds__(FUSED ? kFusedThreads : kTcThreads, 1)
 tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA0, const __grid_constant__ CUtensorMap tmA1,
                const __grid_constant__ CUtensorMap tmB0, const __grid_constant__ CUtensorMap tmB1,
@@ -384,6 +387,7 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA0, const __grid_constant__
       for (int c = 0; c < unit_chunks && ok; ++c, ++gchunk) {
         const int r_main = (NTERMS == 1) ? (int)(gchunk & 1) : 0;
         const bool with_x = (NTERMS == 3) && (p.order == 1);
+        constexpr bool reordered = (NTERMS == 3) && REORD;
         {
           SGC_T0();
           if (!wait_tfull(r_main)) { ok = false; break; }
@@ -394,6 +398,35 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA0, const __grid_constant__
         tc_fence_after_sync();
         const uint32_t t_main = tmem_base + lane_addr + r_main * kBN + half * 128;
         const uint32_t t_x = tmem_base + lane_addr + kBN + half * 128;
+        if constexpr (reordered) {
+          // Reordered elementwise (Sec. 4.5, last paragraph): the block's corrections, already
+          // summed at their own scale, are scaled and added to the block's hi*hi product, and the
+          // accumulator takes the block once:  acc = acc + (P_x / s_f + P_hh).
+          if (!wait_tfull(1)) { ok = false; break; }
+          tc_fence_after_sync();
+          constexpr int GR = 16;
+#pragma unroll
+          for (int g = 0; g < 128 / GR; ++g) {
+            uint32_t vh[GR], vx[GR];
+            tmem_ld_cols(t_main + g * GR, vh);
+            tmem_ld_cols(t_x + g * GR, vx);
+            tmem_ld_wait();
+#pragma unroll
+            for (int j = 0; j < GR; ++j) {
+              const float block =
+                  __fadd_rn(__fmul_rn(__uint_as_float(vx[j]), p.inv_scale), __uint_as_float(vh[j]));
+              S[g * GR + j] = (c == 0) ? block : __fadd_rn(S[g * GR + j], block);
+            }
+          }
+          tc_fence_before_sync();
+          __syncwarp();
+          if (lane == 0) {
+            arrive_tempty(r_main);
+            arrive_tempty(1);
+          }
+          drains[r_main]++;
+          drains[1]++;
+        } else {
 #pragma unroll
         for (int g = 0; g < 128 / GW; ++g) {
           uint32_t v[GW];
@@ -431,6 +464,7 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA0, const __grid_constant__
           if (lane == 0) arrive_tempty(1);
           drains[1]++;
         }
+        }  // not reordered
         SGC_TADD(7, blockIdx.x == 0 && threadIdx.x == 0);
         SGC_TADD(14, blockIdx.x == 1 && threadIdx.x == 0);
       }
@@ -577,7 +611,7 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA0, const __grid_constant__
           const int kb_end = min(kb1, kb_begin + chunk);
           // Region(s) this k-block accumulates into, and which of them start from zero here.
           const int r_main = (NTERMS == 1) ? (int)(gchunk & 1) : 0;
-          const bool x_fresh = (NTERMS == 3) && (p.order == 1 || c == 0);
+          const bool x_fresh = (NTERMS == 3) && (p.order != 0 || c == 0);
           bool main_ready = false, x_ready = !x_fresh;
           const uint32_t d_x = tmem_base + kBN;
           const uint32_t d_main = tmem_base + r_main * kBN;
@@ -683,7 +717,7 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA0, const __grid_constant__
               continue;
             }
 #endif
-            if (NTERMS == 3 && p.order == 1) {
+            if (NTERMS == 3 && p.order != 0) {
               // Elementwise: both regions go to the accumulate warps after every k-block.  hi*hi
               // first and handed over at once: it is drained while the correction products run,
               // and the corrections are drained while the next block's hi*hi products run.
@@ -707,7 +741,7 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA0, const __grid_constant__
             commit_both(&tfull_bar[r_main]);
             fills[r_main]++;
           }
-          if (NTERMS == 3 && (p.order == 1 || c == unit_chunks - 1)) {
+          if (NTERMS == 3 && (p.order != 0 || c == unit_chunks - 1)) {
             commit_both(&tfull_bar[1]);
             fills[1]++;
           }

@@ -108,7 +108,11 @@ int set_kernel_attrs(sgemm_cube_ctx* h) {
       cudaFuncSetAttribute(sgc::tc_gemm_kernel<3, true, false>, attr, (int)sgc::TcCfg<3, false, true>::SMEM_BYTES) != cudaSuccess ||
       cudaFuncSetAttribute(sgc::tc_gemm_kernel<1, false, true>, attr, (int)sgc::TcCfg<1, true>::SMEM_BYTES) != cudaSuccess ||
       cudaFuncSetAttribute(sgc::tc_gemm_kernel<3, false, true>, attr, (int)sgc::TcCfg<3, true>::SMEM_BYTES) != cudaSuccess ||
-      cudaFuncSetAttribute(sgc::tc_gemm_kernel<3, true, true>, attr, (int)sgc::TcCfg<3, true, true>::SMEM_BYTES) != cudaSuccess) {
+      cudaFuncSetAttribute(sgc::tc_gemm_kernel<3, true, true>, attr, (int)sgc::TcCfg<3, true, true>::SMEM_BYTES) != cudaSuccess ||
+      cudaFuncSetAttribute(sgc::tc_gemm_kernel<3, false, false, true>, attr, (int)sgc::TcCfg<3, false>::SMEM_BYTES) != cudaSuccess ||
+      cudaFuncSetAttribute(sgc::tc_gemm_kernel<3, true, false, true>, attr, (int)sgc::TcCfg<3, false, true>::SMEM_BYTES) != cudaSuccess ||
+      cudaFuncSetAttribute(sgc::tc_gemm_kernel<3, false, true, true>, attr, (int)sgc::TcCfg<3, true>::SMEM_BYTES) != cudaSuccess ||
+      cudaFuncSetAttribute(sgc::tc_gemm_kernel<3, true, true, true>, attr, (int)sgc::TcCfg<3, true, true>::SMEM_BYTES) != cudaSuccess) {
     cudaGetLastError();
     return SGEMM_CUBE_CUDA_ERROR;
   }
@@ -128,12 +132,12 @@ bool use_pair(const sgemm_cube_ctx* h, int M, int N, bool fused) {
 }
 
 // Launch one tensor-core kernel: a persistent grid of single CTAs, or of 2-CTA clusters (PAIR).
-template <int NTERMS, bool FUSED, bool PAIR>
-int launch_tc_kernel(sgemm_cube_ctx* h, int M, int N, const CUtensorMap& tmA0, const CUtensorMap& tmA1,
-                     const CUtensorMap& tmB0, const CUtensorMap& tmB1, const sgc::TcGemmParams& p,
-                     cudaStream_t st) {
+template <int NTERMS, bool FUSED, bool PAIR, bool REORD>
+int launch_tc_kernel_impl(sgemm_cube_ctx* h, int M, int N, const CUtensorMap& tmA0, const CUtensorMap& tmA1,
+                          const CUtensorMap& tmB0, const CUtensorMap& tmB1, const sgc::TcGemmParams& p,
+                          cudaStream_t st) {
   using Cfg = sgc::TcCfg<NTERMS, PAIR, FUSED>;
-  auto kernel = sgc::tc_gemm_kernel<NTERMS, FUSED, PAIR>;
+  auto kernel = sgc::tc_gemm_kernel<NTERMS, FUSED, PAIR, REORD>;
   cudaLaunchConfig_t cfg;
   memset(&cfg, 0, sizeof(cfg));
   cfg.blockDim = dim3(FUSED ? sgc::kFusedThreads : sgc::kTcThreads, 1, 1);
@@ -167,6 +171,18 @@ int launch_tc_kernel(sgemm_cube_ctx* h, int M, int N, const CUtensorMap& tmA0, c
   h->launches++;
   return cudaLaunchKernelEx(&cfg, kernel, tmA0, tmA1, tmB0, tmB1, p) == cudaSuccess
              ? SGEMM_CUBE_OK : (cudaGetLastError(), SGEMM_CUBE_CUDA_ERROR);
+}
+
+// The reordered elementwise order (p.order == 2) runs its own instantiation of the kernel.
+template <int NTERMS, bool FUSED, bool PAIR>
+int launch_tc_kernel(sgemm_cube_ctx* h, int M, int N, const CUtensorMap& tmA0, const CUtensorMap& tmA1,
+                     const CUtensorMap& tmB0, const CUtensorMap& tmB1, const sgc::TcGemmParams& p,
+                     cudaStream_t st) {
+  if constexpr (NTERMS == 3) {
+    if (p.order == SGEMM_CUBE_ELEMENTWISE_REORDERED)
+      return launch_tc_kernel_impl<NTERMS, FUSED, PAIR, true>(h, M, N, tmA0, tmA1, tmB0, tmB1, p, st);
+  }
+  return launch_tc_kernel_impl<NTERMS, FUSED, PAIR, false>(h, M, N, tmA0, tmA1, tmB0, tmB1, p, st);
 }
 
 // Dimensions may be zero (an empty operand may then be a null pointer); negative ones are errors.
@@ -564,7 +580,7 @@ int sgemm_cube(sgemm_cube_handle h, int M, int N, int K, const float* A, int64_t
   if (rc) return rc;
   if (missing_operand(M, N, K, A, A, B, B, C)) return SGEMM_CUBE_INVALID_ARG;
   if (scale_exp < 0 || scale_exp > 24) return SGEMM_CUBE_INVALID_ARG;
-  if (order != SGEMM_CUBE_TERMWISE && order != SGEMM_CUBE_ELEMENTWISE) return SGEMM_CUBE_INVALID_ARG;
+  if (order < SGEMM_CUBE_TERMWISE || order > SGEMM_CUBE_ELEMENTWISE_REORDERED) return SGEMM_CUBE_INVALID_ARG;
   DeviceGuard g(h->device);
   if (!g.ok) return SGEMM_CUBE_CUDA_ERROR;
   if (empty_problem(M, N, K, C, ldc, static_cast<cudaStream_t>(stream), false, false, &rc)) return rc;
@@ -581,7 +597,7 @@ int sgemm_cube_presplit(sgemm_cube_handle h, int M, int N, int K, const uint16_t
   if (rc) return rc;
   if (missing_operand(M, N, K, Ahi, Alo, Bhi, Blo, C)) return SGEMM_CUBE_INVALID_ARG;
   if (scale_exp < 0 || scale_exp > 24) return SGEMM_CUBE_INVALID_ARG;
-  if (order != SGEMM_CUBE_TERMWISE && order != SGEMM_CUBE_ELEMENTWISE) return SGEMM_CUBE_INVALID_ARG;
+  if (order < SGEMM_CUBE_TERMWISE || order > SGEMM_CUBE_ELEMENTWISE_REORDERED) return SGEMM_CUBE_INVALID_ARG;
   DeviceGuard g(h->device);
   if (!g.ok) return SGEMM_CUBE_CUDA_ERROR;
   if (empty_problem(M, N, K, C, ldc, static_cast<cudaStream_t>(stream), false, false, &rc)) return rc;
@@ -696,7 +712,7 @@ int sgemm_cube_host(sgemm_cube_handle h, int M, int N, int K, const float* A_hos
   if (rc) return rc;
   if (missing_operand(M, N, K, A_host, A_host, B_host, B_host, C_host)) return SGEMM_CUBE_INVALID_ARG;
   if (scale_exp < 0 || scale_exp > 24) return SGEMM_CUBE_INVALID_ARG;
-  if (order != SGEMM_CUBE_TERMWISE && order != SGEMM_CUBE_ELEMENTWISE) return SGEMM_CUBE_INVALID_ARG;
+  if (order < SGEMM_CUBE_TERMWISE || order > SGEMM_CUBE_ELEMENTWISE_REORDERED) return SGEMM_CUBE_INVALID_ARG;
   DeviceGuard g(h->device);
   if (!g.ok) return SGEMM_CUBE_CUDA_ERROR;
   if (empty_problem(M, N, K, C_host, ldc, static_cast<cudaStream_t>(stream), true, false, &rc)) return rc;
@@ -924,7 +940,7 @@ int sgemm_cube_scaled(sgemm_cube_handle h, int M, int N, int K, const float* A, 
   if (rc) return rc;
   if (missing_operand(M, N, K, A, A, B, B, C)) return SGEMM_CUBE_INVALID_ARG;
   if (scale_exp < 0 || scale_exp > 24) return SGEMM_CUBE_INVALID_ARG;
-  if (order != SGEMM_CUBE_TERMWISE && order != SGEMM_CUBE_ELEMENTWISE) return SGEMM_CUBE_INVALID_ARG;
+  if (order < SGEMM_CUBE_TERMWISE || order > SGEMM_CUBE_ELEMENTWISE_REORDERED) return SGEMM_CUBE_INVALID_ARG;
   if (p_a < -126 || p_a > 126 || p_b < -126 || p_b > 126) return SGEMM_CUBE_INVALID_ARG;
   DeviceGuard g(h->device);
   if (!g.ok) return SGEMM_CUBE_CUDA_ERROR;

@@ -10,7 +10,7 @@ U32 = 2.0 ** -24
 # k-block lengths the library uses by default (include/sgemm_cube.h, SGEMM_CUBE_OPT_*); the
 # oracle is run with the same block length so that both sides realise the same Eq. termwise /
 # Eq. elementwise bracketing.
-K_BLOCK = {binding.TERMWISE: 128, binding.ELEMENTWISE: 64}
+K_BLOCK = {binding.TERMWISE: 128, binding.ELEMENTWISE: 64, binding.ELEMENTWISE_REORDERED: 64}
 
 
 def to_dev(x):

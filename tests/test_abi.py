@@ -84,6 +84,7 @@ def test_binding_constants_match_the_header():
              "SGEMM_CUBE_UNSUPPORTED_ARCH": binding.UNSUPPORTED_ARCH,
              "SGEMM_CUBE_ALLOC_FAILED": binding.ALLOC_FAILED, "SGEMM_CUBE_TOO_LARGE": binding.TOO_LARGE,
              "SGEMM_CUBE_TERMWISE": binding.TERMWISE, "SGEMM_CUBE_ELEMENTWISE": binding.ELEMENTWISE,
+             "SGEMM_CUBE_ELEMENTWISE_REORDERED": binding.ELEMENTWISE_REORDERED,
              "SGEMM_CUBE_OPT_TERMWISE_K_BLOCK": binding.OPT_TERMWISE_K_BLOCK,
              "SGEMM_CUBE_OPT_ELEMENTWISE_K_BLOCK": binding.OPT_ELEMENTWISE_K_BLOCK,
              "SGEMM_CUBE_OPT_CTA_PAIR": binding.OPT_CTA_PAIR, "SGEMM_CUBE_OPT_STRATEGY": binding.OPT_STRATEGY,

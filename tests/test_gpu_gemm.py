@@ -392,6 +392,44 @@ def test_special_values_propagate_like_the_oracle(handle, path, order):
           label="rows and columns without special values")
 
 
+R = binding.ELEMENTWISE_REORDERED
+
+
+@pytest.mark.parametrize("path", ["fused", "two_phase", "presplit"])
+@pytest.mark.parametrize("shape", [(129, 257, 33), (300, 520, 200), (512, 768, 1000), (1024, 1024, 4096)])
+def test_reordered_elementwise_order(handle, path, shape):
+    M, N, K = shape
+    A, B = inputs.make_pair("normal", 17, M, N, K)
+    C = run(handle, path, padded_dev(A, 4), padded_dev(B, 4), 11, R)
+    gates(C, A, B, 11, R, label="reordered %s %s" % (path, shape))
+    # one-signed data: same gates
+    A2 = inputs.uniform_range(3, (M, K), 0, True, stream=0)
+    B2 = inputs.uniform_range(3, (K, N), 0, True, stream=1)
+    gates(run(handle, path, padded_dev(A2, 4), padded_dev(B2, 4), 11, R), A2, B2, 11, R, label="nonneg")
+
+
+def test_reordered_elementwise_keeps_what_a_block_adds_up_to(handle):
+    # Block 0 makes the accumulator 2^10 (ulp 2^-13).  Block 1 holds hi*hi = 2^-14 (1 - 2^-20),
+    # just under half an ulp, and a correction of 2^-29: added one after the other to the
+    # accumulator both are lost (Eq. elementwise, also as the kernel realises it); added
+    # together first they exceed half an ulp and the sum rounds up (Sec. 4.5, last paragraph).
+    a_hi = 2.0 ** -7 * (1 + 2.0 ** -10)
+    b = 2.0 ** -7 * (1 - 2.0 ** -10)
+    a = a_hi + 2.0 ** -22                      # residual 2^-22, far inside half an FP16 ulp
+    A = np.zeros((128, 128), dtype=np.float32)
+    B = np.zeros((128, 256), dtype=np.float32)
+    A[:, 0], B[0, :] = 32.0, 32.0
+    A[:, 64], B[64, :] = a, b
+    assert float(A[0, 64]) == a and float(B[64, 0]) == b
+    for path in ("fused", "two_phase"):
+        el = run(handle, path, to_dev(A), to_dev(B), 11, E)
+        ro = run(handle, path, to_dev(A), to_dev(B), 11, R)
+        assert np.all(el == np.float32(1024.0))
+        assert np.all(ro == np.float32(1024.0 + 2.0 ** -13))
+        assert np.array_equal(ro, oracle.sgemm_cube(A, B, 11, R, 64))
+        assert np.array_equal(el, oracle.sgemm_cube(A, B, 11, E, 64))
+
+
 def test_hgemm_matches_fp64_product_of_fp16_inputs(handle):
     for (M, N, K) in [(128, 256, 64), (200, 300, 136), (1024, 1024, 1024)]:
         A = inputs.normal(1, (M, (K + 7) // 8 * 8))[:, :K]

@@ -27,7 +27,7 @@ def test_variants_agree_bitwise_on_random_configurations(seed):
             N = rng.choice([1, 8, 100, 255, 256, 257, 512, 640, 1000, 1536])
             K = rng.choice([1, 16, 63, 64, 65, 128, 200, 512, 1000, 2048, 4100])
             kbt, kbe = rng.choice([64, 128, 256, 512]), rng.choice([64, 128, 256])
-            order = rng.choice([binding.TERMWISE, binding.ELEMENTWISE])
+            order = rng.choice([binding.TERMWISE, binding.ELEMENTWISE, binding.ELEMENTWISE_REORDERED])
             h.sgemm_cube_set_option(binding.OPT_TERMWISE_K_BLOCK, kbt)
             h.sgemm_cube_set_option(binding.OPT_ELEMENTWISE_K_BLOCK, kbe)
             g = torch.Generator(device="cuda:0")

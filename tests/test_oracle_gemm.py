@@ -184,6 +184,24 @@ def test_reordered_elementwise_keeps_what_the_plain_order_loses_inside_a_block()
         assert np.array_equal(got, _brute_force(A, B, 11, order, 1))
 
 
+def test_reordered_elementwise_adds_a_block_to_the_accumulator_once():
+    # Accumulator 2^10 (ulp 2^-13) after block 0; block 1 holds hi*hi = 2^-14 (1 - 2^-20), just
+    # under half an ulp, and a correction of about 2^-29.  Eq. elementwise adds them one by one
+    # and loses both; the termwise hi*hi stream loses the product as well; the reordered order
+    # adds the block's own sum, which exceeds half an ulp, and rounds up.
+    a_hi = 2.0 ** -7 * (1 + 2.0 ** -10)
+    b = 2.0 ** -7 * (1 - 2.0 ** -10)
+    a = a_hi + 2.0 ** -22
+    A = np.array([[32.0, a]], dtype=np.float32)
+    B = np.array([[32.0], [b]], dtype=np.float32)
+    res = {o: float(oracle.sgemm_cube(A, B, s=11, order=o, kb=1)[0, 0])
+           for o in (oracle.TERMWISE, oracle.ELEMENTWISE, oracle.ELEMENTWISE_REORDERED)}
+    assert res[oracle.TERMWISE] == 1024.0 and res[oracle.ELEMENTWISE] == 1024.0
+    assert res[oracle.ELEMENTWISE_REORDERED] == 1024.0 + 2.0 ** -13
+    exact = 1024.0 + float(A[0, 1]) * float(B[1, 0])
+    assert abs(res[oracle.ELEMENTWISE_REORDERED] - exact) < abs(res[oracle.TERMWISE] - exact)
+
+
 @pytest.mark.parametrize("kind", ["uniform_pm1", "exponent_spread", "normal"])
 @pytest.mark.parametrize("K", [15, 64, 300])
 def test_main_bound_holds_entrywise_for_termwise(kind, K):

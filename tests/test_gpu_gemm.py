@@ -463,7 +463,8 @@ def test_argument_errors(handle):
     assert call(lda=15) == binding.INVALID_ARG
     assert call(ldc=7) == binding.INVALID_ARG
     assert call(s=25) == binding.INVALID_ARG
-    assert call(order=2) == binding.INVALID_ARG
+    assert call(order=3) == binding.INVALID_ARG and call(order=-1) == binding.INVALID_ARG
+    assert call(order=2) == binding.OK                       # the reordered elementwise order
     assert call(A=None) == binding.INVALID_ARG
     assert call(A=p(A) + 4) == binding.MISALIGNED
     assert call(lda=18) == binding.MISALIGNED

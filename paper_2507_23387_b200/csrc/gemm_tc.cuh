@@ -915,7 +915,7 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA0, const __grid_constant__
       // Generic-proxy stores must be visible to the tensor core (async proxy) before the hand-over.
       {
         SGC_T0();
-        if (PAIR) fence_proxy_async_all();
+        if (PAIR) fence_proxy_async_smem_cluster();
         else fence_proxy_async_smem();
         __syncwarp();
         if (lane == 0) {

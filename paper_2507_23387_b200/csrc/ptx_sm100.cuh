@@ -266,6 +266,11 @@ __device__ __forceinline__ bool mbar_wait_bounded_cluster(uint64_t* bar, uint32_
 __device__ __forceinline__ void fence_proxy_async_all() {
   asm volatile("fence.proxy.async;" ::: "memory");
 }
+// Generic-proxy writes to shared memory made visible to the async proxy of every CTA of the
+// cluster (in a CTA pair the peer's tensor core reads this CTA's half of the B tile).
+__device__ __forceinline__ void fence_proxy_async_smem_cluster() {
+  asm volatile("fence.proxy.async.shared::cluster;" ::: "memory");
+}
 // 2-D tiled load into this CTA's shared memory whose completion bytes are counted on the
 // mbarrier at the same offset in the LEADER CTA (bit 24 of a shared::cluster address holds the
 // CTA rank inside a pair).  The data itself goes to the issuing CTA only.

@@ -354,8 +354,13 @@ int launch_tc_gemm(sgemm_cube_ctx* h, int M, int N, int K, const uint16_t* Ahi, 
     h->launches++;
     return cudaGetLastError() == cudaSuccess ? SGEMM_CUBE_OK : SGEMM_CUBE_CUDA_ERROR;
   }
-  return pair ? launch_tc_kernel<NTERMS, false, true>(h, M, N, tmA0, tmA1, tmB0, tmB1, p, st)
-                           : launch_tc_kernel<NTERMS, false, false>(h, M, N, tmA0, tmA1, tmB0, tmB1, p, st);
+  if (pair) {
+    rc = launch_tc_kernel<NTERMS, false, true>(h, M, N, tmA0, tmA1, tmB0, tmB1, p, st);
+    // Clusters that cannot be scheduled (a partitioned or partly occupied device): when the pair
+    // mode was the library's own choice, single CTAs compute the same bits.
+    if (rc != SGEMM_CUBE_CUDA_ERROR || h->cta_pair != 2) return rc;
+  }
+  return launch_tc_kernel<NTERMS, false, false>(h, M, N, tmA0, tmA1, tmB0, tmB1, p, st);
 }
 
 int launch_fused(sgemm_cube_ctx* h, int M, int N, int K, const float* A, int64_t lda, const float* B,

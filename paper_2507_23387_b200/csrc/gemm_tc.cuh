@@ -14,11 +14,11 @@
 //                round-to-nearest into running sums held in registers, form C, store it
 //   not FUSED (384 threads): warp 8 = TMA producer (FP16 tiles global -> shared, swizzled UMMA
 //                layout), warp 9 = MMA issuer
-//   FUSED (512 threads): warps 8-14 = converter warps: FP32 tiles global -> registers -> (hi, lo)
-//                FP16 words -> shared memory, written directly in the swizzled UMMA layout;
-//                warp 15 = MMA issuer.  The FP32 data never touches shared memory: with
-//                128 bytes/clk of shared-memory bandwidth per SM the tensor core's own operand
-//                reads leave no room for an FP32 staging round trip.
+//   FUSED (512 threads): warp 13 = TMA producer staging FP32 tiles of A and B in a shared-memory
+//                ring (128-byte swizzle); warps 8-11 = converter warps: FP32 ring -> registers ->
+//                (hi, lo) FP16 words -> the FP16 ring, written directly in the swizzled UMMA
+//                layout; warp 12 = MMA issuer.  Every converter thread works on the same tile
+//                positions in every stage, so its shared-memory offsets are constants.
 //   The MMA issuer is one thread issuing tcgen05.mma kind::f16 (M = 128, N = 256, K = 16).
 //
 // Why the running sums live in registers.  The tensor core adds products into its FP32
@@ -37,6 +37,8 @@
 
 #include <cuda_fp16.h>
 
+#include <type_traits>
+
 #include "ptx_sm100.cuh"
 
 namespace sgc {
@@ -45,9 +47,12 @@ constexpr int kBM = 128;            // CTA tile rows  (UMMA M)
 constexpr int kBN = 256;            // CTA tile cols  (UMMA N)
 constexpr int kNumEpiWarps = 8;     // warps 0-7
 constexpr int kTcThreads = 384;     // not FUSED: + TMA warp + MMA warp (+ 2 idle warps: whole warpgroup)
-constexpr int kFusedThreads = 512;  // FUSED: + 7 converter warps + MMA warp
-constexpr int kNumConvWarps = 7;
-constexpr int kConvThreads = kNumConvWarps * 32;   // 224
+#ifndef SGC_CONV_WARPS
+#define SGC_CONV_WARPS 4
+#endif
+constexpr int kNumConvWarps = SGC_CONV_WARPS;      // a multiple of 4 (see the converter role)
+// FUSED: + converter warps + MMA warp + TMA warp, rounded up to whole warpgroups
+constexpr int kFusedThreads = ((kNumEpiWarps + kNumConvWarps + 2 + 3) / 4) * 128;
 constexpr uint32_t kTmemCols = 512;
 
 // error codes written to the device error word (which wait gave up)
@@ -58,6 +63,7 @@ enum : unsigned int {
   kErrEpiTmemFullWait = 0x104,
   kErrDrainWait = 0x105,
   kErrConvEmptyWait = 0x106,
+  kErrConvFullWait = 0x107,
 };
 
 // Optional role timing (compile with -DSGC_ROLE_TIMING): CTA 0 adds the clocks each role spends in
@@ -117,10 +123,18 @@ struct TcCfg {
   static constexpr uint32_t A_TILE = kBM * BK * 2;        // one FP16 A tile
   static constexpr uint32_t B_TILE = BK * BN_CTA * 2;     // one FP16 B tile (this CTA's columns)
   static constexpr uint32_t STAGE_BYTES = (NTERMS == 1) ? (A_TILE + B_TILE) : 2 * (A_TILE + B_TILE);
-  static constexpr int STAGES = (196608 / STAGE_BYTES) > 8 ? 8 : (196608 / STAGE_BYTES);
+  // FUSED: a second ring holds the FP32 tiles that TMA stages for the converter warps (same k
+  // depth, same bytes per stage as the (hi, lo) pair it becomes); the two rings share the space.
+  static constexpr uint32_t A32_TILE = FUSED ? kBM * BK * 4 : 0;
+  static constexpr uint32_t B32_TILE = FUSED ? BK * BN_CTA * 4 : 0;   // BN_CTA / 32 boxes of 32 columns
+  static constexpr uint32_t STAGE32_BYTES = A32_TILE + B32_TILE;
+  static constexpr int STAGES = FUSED ? (int)(196608 / (STAGE_BYTES + STAGE32_BYTES))
+                                      : ((196608 / STAGE_BYTES) > 8 ? 8 : (int)(196608 / STAGE_BYTES));
+  static constexpr int STAGES32 = FUSED ? STAGES : 0;
+  static constexpr uint32_t RING_BYTES = STAGES * STAGE_BYTES + STAGES32 * STAGE32_BYTES;
   static constexpr uint32_t STORE_STAGING = kNumEpiWarps * 4096;   // 32 rows x 128 bytes per warp
   static constexpr uint32_t SMEM_BYTES =
-      STAGES * STAGE_BYTES + 1024 /*align*/ + 256 /*barriers*/ + STORE_STAGING;
+      RING_BYTES + 1024 /*align*/ + 256 /*barriers*/ + STORE_STAGING;
 };
 
 // Tile rasterisation: groups of `group_m` tile-rows are walked column by column so that the CTAs
@@ -164,13 +178,20 @@ __device__ __forceinline__ void store16(float* D, long long ldd, int M, int N, i
 }
 
 // ------------------------------------------------------------------------------------------
-// Converter-warp helpers (FUSED).  One "item" is 8 consecutive FP32 elements of a row (32 bytes
-// in, one 16-byte chunk of the hi tile and one of the lo tile out).
-struct ConvItem { float4 a, b; };
+// Converter-warp helpers (FUSED).  One "item" is 8 consecutive FP32 elements of a tile row: two
+// 16-byte chunks of the FP32 ring in, one 16-byte chunk of the hi tile and one of the lo tile out.
+struct ConvScale {
+  float scale;            // 2^s
+  uint64_t scale2;        // {2^s, 2^s} packed
+  uint16_t neg_scale_h;   // -2^s as FP16 (valid when fast)
+  bool fast;              // s <= 15
+};
 
-__device__ __forceinline__ void split_pair(float x0, float x1, float scale, uint32_t& hi2,
-                                           uint32_t& lo2) {
-  // hi = fl16(x); lo = fl16((x - hi) * 2^s): the subtraction and the scaling are exact (Sec. 3.3).
+// Two elements, plain form:  hi = fl16(x); lo = fl16((x - hi) * 2^s); the subtraction and the
+// scaling are exact (Sec. 3.3).
+__device__ __forceinline__ void split_pair(uint64_t xp, float scale, uint32_t& hi2, uint32_t& lo2) {
+  float x0, x1;
+  asm("mov.b64 {%0, %1}, %2;" : "=f"(x0), "=f"(x1) : "l"(xp));
   const __half2 h = __floats2half2_rn(x0, x1);
   const float2 hf = __half22float2(h);
   const __half2 l = __floats2half2_rn(__fmul_rn(__fsub_rn(x0, hf.x), scale),
@@ -179,18 +200,21 @@ __device__ __forceinline__ void split_pair(float x0, float x1, float scale, uint
   lo2 = *reinterpret_cast<const uint32_t*>(&l);
 }
 
-// Same words with fewer instructions, for s <= 15 (2^s representable in FP16):
-//   xs = x * 2^s            one packed FP32x2 multiply for the pair (exact)
+// The same words in five instructions per pair, for s <= 15 (2^s representable in FP16):
+//   hi = cvt.f16x2(x)       packed conversion
+//   xs = x * 2^s            one packed FP32x2 multiply (exact)
 //   t  = hi * (-2^s) + xs   one mixed-precision FMA per element (FP16 x FP16 + FP32): the exact value
 //                           (x - hi) * 2^s is representable, so the single rounding changes nothing
-// which avoids widening hi to FP32 and the separate subtraction.  (For |x| >= 2^(128-s), outside
-// the method's range, xs overflows and lo becomes NaN where the plain form gives inf.)
-__device__ __forceinline__ void split_pair_fast(float x0, float x1, uint64_t scale2,
-                                                uint16_t neg_scale_h, uint32_t& hi2, uint32_t& lo2) {
+//   lo = cvt.f16x2(t)
+// (For |x| >= 2^(128-s), outside the method's range, xs overflows and lo becomes NaN where the
+// plain form gives inf.)
+__device__ __forceinline__ void split_pair_fast(uint64_t xp, uint64_t scale2, uint16_t neg_scale_h,
+                                                uint32_t& hi2, uint32_t& lo2) {
+  float x0, x1;
+  asm("mov.b64 {%0, %1}, %2;" : "=f"(x0), "=f"(x1) : "l"(xp));
   uint32_t h;
   asm("cvt.rn.f16x2.f32 %0, %1, %2;" : "=r"(h) : "f"(x1), "f"(x0));
-  uint64_t xp, xs;
-  asm("mov.b64 %0, {%1, %2};" : "=l"(xp) : "f"(x0), "f"(x1));
+  uint64_t xs;
   asm("mul.rn.f32x2 %0, %1, %2;" : "=l"(xs) : "l"(xp), "l"(scale2));
   float xs0, xs1, t0, t1;
   asm("mov.b64 {%0, %1}, %2;" : "=f"(xs0), "=f"(xs1) : "l"(xs));
@@ -204,52 +228,30 @@ __device__ __forceinline__ void split_pair_fast(float x0, float x1, uint64_t sca
   lo2 = l;
 }
 
-struct ConvScale {
-  float scale;            // 2^s
-  uint64_t scale2;        // {2^s, 2^s} packed
-  uint16_t neg_scale_h;   // -2^s as FP16 (valid when fast)
-  bool fast;              // s <= 15
-};
-
-__device__ __forceinline__ void convert_store(const ConvItem& it, const ConvScale& cs,
-                                              uint32_t hi_addr, uint32_t lo_addr) {
+// One item: FP32 chunks at shared addresses src0 / src1 (elements 0-3 / 4-7) -> hi chunk at dst,
+// lo chunk at dst + lo_off.
+template <bool FAST>
+__device__ __forceinline__ void convert_item(uint32_t src0, uint32_t src1, uint32_t dst, uint32_t lo_off,
+                                             const ConvScale& cs) {
+  uint64_t x01, x23, x45, x67;
+  asm volatile("ld.shared.v2.b64 {%0, %1}, [%2];" : "=l"(x01), "=l"(x23) : "r"(src0) : "memory");
+  asm volatile("ld.shared.v2.b64 {%0, %1}, [%2];" : "=l"(x45), "=l"(x67) : "r"(src1) : "memory");
   uint4 h, l;
-  if (cs.fast) {
-    split_pair_fast(it.a.x, it.a.y, cs.scale2, cs.neg_scale_h, h.x, l.x);
-    split_pair_fast(it.a.z, it.a.w, cs.scale2, cs.neg_scale_h, h.y, l.y);
-    split_pair_fast(it.b.x, it.b.y, cs.scale2, cs.neg_scale_h, h.z, l.z);
-    split_pair_fast(it.b.z, it.b.w, cs.scale2, cs.neg_scale_h, h.w, l.w);
+  if (FAST) {
+    split_pair_fast(x01, cs.scale2, cs.neg_scale_h, h.x, l.x);
+    split_pair_fast(x23, cs.scale2, cs.neg_scale_h, h.y, l.y);
+    split_pair_fast(x45, cs.scale2, cs.neg_scale_h, h.z, l.z);
+    split_pair_fast(x67, cs.scale2, cs.neg_scale_h, h.w, l.w);
   } else {
-    const float scale = cs.scale;
-    split_pair(it.a.x, it.a.y, scale, h.x, l.x);
-    split_pair(it.a.z, it.a.w, scale, h.y, l.y);
-    split_pair(it.b.x, it.b.y, scale, h.z, l.z);
-    split_pair(it.b.z, it.b.w, scale, h.w, l.w);
+    split_pair(x01, cs.scale, h.x, l.x);
+    split_pair(x23, cs.scale, h.y, l.y);
+    split_pair(x45, cs.scale, h.z, l.z);
+    split_pair(x67, cs.scale, h.w, l.w);
   }
-  asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(hi_addr), "r"(h.x), "r"(h.y),
+  asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(dst), "r"(h.x), "r"(h.y),
                "r"(h.z), "r"(h.w) : "memory");
-  asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(lo_addr), "r"(l.x), "r"(l.y),
+  asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(dst + lo_off), "r"(l.x), "r"(l.y),
                "r"(l.z), "r"(l.w) : "memory");
-}
-
-// 8 elements of row `row` starting at column `col` of a rows x cols row-major matrix; elements
-// outside the matrix read as zero (split(0) = (0, 0), so zero padding is exact).
-__device__ __forceinline__ ConvItem load_item_guarded(const float* __restrict__ X, long long ld,
-                                                      int rows, int cols, int row, int col) {
-  ConvItem it;
-  if (row < rows && col + 8 <= cols) {
-    const float4* src = reinterpret_cast<const float4*>(X + (long long)row * ld + col);
-    it.a = __ldg(src);
-    it.b = __ldg(src + 1);
-  } else {
-    float v[8];
-#pragma unroll
-    for (int j = 0; j < 8; ++j)
-      v[j] = (row < rows && col + j < cols) ? __ldg(X + (long long)row * ld + col + j) : 0.f;
-    it.a = make_float4(v[0], v[1], v[2], v[3]);
-    it.b = make_float4(v[4], v[5], v[6], v[7]);
-  }
-  return it;
 }
 
 __device__ __forceinline__ void tmem_ld_cols(uint32_t taddr, uint32_t (&r)[16]) { tmem_ld_32x32b_x16(taddr, r); }
@@ -274,8 +276,10 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA0, const __grid_constant__
   // leader and are signalled by both CTAs, while its commits arrive on the barriers of both.
   const uint32_t cta_rank = PAIR ? cluster_ctarank() : 0u;
   const bool leader = (cta_rank == 0);
-  constexpr int kProducerWarp = 8;                    // not FUSED
-  constexpr int kMmaWarp = FUSED ? 15 : 9;
+  // not FUSED: warp 8 loads FP16 tiles; FUSED: the warp after the MMA warp loads FP32 tiles
+  constexpr int kMmaWarp = FUSED ? kNumEpiWarps + kNumConvWarps : 9;
+  constexpr int kProducerWarp = FUSED ? kMmaWarp + 1 : 8;
+  constexpr int STAGES32 = Cfg::STAGES32;
   static_assert(!FUSED || NTERMS == 3, "the fused kernel computes all three products");
 
   extern __shared__ uint8_t smem_raw[];
@@ -283,15 +287,22 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA0, const __grid_constant__
   // of the shared-memory address bits, so every tile must start on a 1024-byte boundary.
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) &
                                              ~uintptr_t(1023));
-  uint64_t* bars = reinterpret_cast<uint64_t*>(smem + STAGES * Cfg::STAGE_BYTES);
+  uint8_t* smem32 = smem + STAGES * Cfg::STAGE_BYTES;       // FUSED: the FP32 ring
+  uint64_t* bars = reinterpret_cast<uint64_t*>(smem + Cfg::RING_BYTES);
   uint64_t* full_bar = bars;                 // [STAGES]  producer/converters -> MMA
   uint64_t* empty_bar = bars + STAGES;       // [STAGES]  MMA -> producer/converters
   uint64_t* tfull_bar = bars + 2 * STAGES;   // [2]       MMA -> epilogue (TMEM region filled)
   uint64_t* tempty_bar = bars + 2 * STAGES + 2;  // [2]   epilogue -> MMA (TMEM region drained)
   uint64_t* drain_bar = bars + 2 * STAGES + 4;   // [1]
-  uint32_t* tmem_base_slot = reinterpret_cast<uint32_t*>(bars + 2 * STAGES + 5);
+  uint64_t* full32_bar = bars + 2 * STAGES + 5;              // [STAGES32]  TMA -> converters
+  uint64_t* empty32_bar = bars + 2 * STAGES + 5 + STAGES32;  // [STAGES32]  converters -> TMA
+  uint32_t* tmem_base_slot = reinterpret_cast<uint32_t*>(bars + 2 * STAGES + 5 + 2 * STAGES32);
   volatile uint32_t* abort_flag = tmem_base_slot + 1;
-  uint8_t* store_staging = smem + STAGES * Cfg::STAGE_BYTES + 256;   // epilogue transposition buffers
+  // PAIR: a wait that gives up also raises the peer's flag (shared::cluster address of the same slot)
+  const uint32_t peer_abort =
+      PAIR ? mapa_u32(smem_u32(tmem_base_slot + 1), cta_rank ^ 1u) : 0u;
+  static_assert((2 * STAGES + 5 + 2 * STAGES32) * 8 + 8 <= 256, "barrier block");
+  uint8_t* store_staging = smem + Cfg::RING_BYTES + 256;   // epilogue transposition buffers
 
   const int warp = threadIdx.x >> 5;
   const int lane = threadIdx.x & 31;
@@ -313,13 +324,17 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA0, const __grid_constant__
       mbar_init(&tfull_bar[r], 1);
       mbar_init(&tempty_bar[r], kNumEpiWarps * (PAIR ? 2 : 1));
     }
+    for (int s = 0; s < STAGES32; ++s) {
+      mbar_init(&full32_bar[s], 1);
+      mbar_init(&empty32_bar[s], kNumConvWarps);
+    }
     mbar_init(drain_bar, 1);
     *abort_flag = 0u;
     fence_mbar_init();
   }
-  if (!FUSED && warp == kProducerWarp && lane == 0) {
+  if (warp == kProducerWarp && lane == 0) {
     tma_prefetch_desc(&tmA0); tma_prefetch_desc(&tmB0);
-    if (NTERMS == 3) { tma_prefetch_desc(&tmA1); tma_prefetch_desc(&tmB1); }
+    if (NTERMS == 3 && !FUSED) { tma_prefetch_desc(&tmA1); tma_prefetch_desc(&tmB1); }
   }
   if (warp == kMmaWarp) {    // whole warp (the same warp in both CTAs of a pair): all 512 TMEM columns
     if (PAIR) { tmem_alloc_pair(tmem_base_slot, kTmemCols); tmem_relinquish_pair(); }
@@ -373,7 +388,7 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA0, const __grid_constant__
     // long as a drain lasts, and the load latency is most of that), 16 where registers are tight.
     constexpr int GW = FUSED ? 16 : 64;
     auto wait_tfull = [&](int r) -> bool {
-      return mbar_wait_bounded(&tfull_bar[r], drains[r] & 1, abort_flag, p.err, kErrEpiTmemFullWait);
+      return mbar_wait_bounded(&tfull_bar[r], drains[r] & 1, abort_flag, p.err, kErrEpiTmemFullWait, peer_abort);
     };
     // "TMEM region drained": arrive on the leader's barrier (the peer does so remotely).
     auto arrive_tempty = [&](int r) {
@@ -575,7 +590,7 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA0, const __grid_constant__
         else umma_commit(bar);
       };
       auto wait = [&](uint64_t* bar, uint32_t parity, unsigned int code) {
-        return PAIR ? mbar_wait_bounded_cluster(bar, parity, abort_flag, p.err, code)
+        return PAIR ? mbar_wait_bounded_cluster(bar, parity, abort_flag, p.err, code, peer_abort)
                     : mbar_wait_bounded(bar, parity, abort_flag, p.err, code);
       };
       constexpr uint64_t a_swz = (Cfg::A_ROW_BYTES == 128) ? kSwizzle128
@@ -682,7 +697,7 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA0, const __grid_constant__
 #ifdef SGC_KLOOK
           constexpr int kLook = SGC_KLOOK;
 #else
-          constexpr int kLook = (((PAIR && FUSED) ? 3 : 2) * 32 + BK - 1) / BK;
+          constexpr int kLook = (2 * 32 + BK - 1) / BK;
 #endif
           if (NTERMS == 3 && p.order == 0 && kb + kLook <= kb_end) {
             // Start of a termwise k-block: the correction products of the first kLook stages go
@@ -752,14 +767,21 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA0, const __grid_constant__
       else umma_commit(drain_bar);
       mbar_wait_bounded(drain_bar, 0, nullptr, p.err, kErrDrainWait);
     }
-  } else if (!FUSED) {
-    setmaxnreg_dec<56>();
-    // ------------------------------------------------------------------ TMA producer (warp 8)
-    if (warp == kProducerWarp && lane == 0) {
+  } else if (warp == kProducerWarp) {
+    if (FUSED) setmaxnreg_dec<88>();
+    else setmaxnreg_dec<56>();
+    // ------------------------------------------------------------------ TMA producer
+    // not FUSED: FP16 operand tiles into the ring the MMA thread reads.  FUSED: FP32 tiles of A
+    // and B into the FP32 ring the converter warps read (this CTA's own rows of A and its own
+    // columns of B; barriers local to the CTA also in a pair).
+    if (lane == 0) {
+      constexpr int RING = FUSED ? STAGES32 : STAGES;
+      uint64_t* const ring_full = FUSED ? full32_bar : full_bar;
+      uint64_t* const ring_empty = FUSED ? empty32_bar : empty_bar;
       uint32_t it = 0;
       bool ok = true;
       auto load = [&](void* dst, const CUtensorMap* map, int x, int y, uint64_t* bar) {
-        if (PAIR) tma_load_2d_pair(dst, map, x, y, bar);    // bytes counted on the leader's barrier
+        if (PAIR && !FUSED) tma_load_2d_pair(dst, map, x, y, bar);   // bytes counted on the leader's barrier
         else tma_load_2d(dst, map, x, y, bar);
       };
       for (int unit = first_tile; unit < num_units && ok; unit += tile_stride) {
@@ -767,150 +789,149 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA0, const __grid_constant__
         unit_rc(unit, tm, tn, kb0, kb1, slice);
         const int n0 = tn * kBN + (PAIR ? (int)cta_rank * Cfg::BN_CTA : 0);   // this CTA's B columns
         for (int kb = kb0; kb < kb1; ++kb, ++it) {
-          const int s = it % STAGES;
-          const uint32_t ph = (it / STAGES) & 1;
-          if (!mbar_wait_bounded(&empty_bar[s], ph ^ 1, abort_flag, p.err, kErrProducerEmptyWait)) {
+          const int s = it % RING;
+          const uint32_t ph = (it / RING) & 1;
+          if (!mbar_wait_bounded(&ring_empty[s], ph ^ 1, abort_flag, p.err, kErrProducerEmptyWait, peer_abort)) {
             ok = false;
             break;
           }
-          uint8_t* st = smem + s * Cfg::STAGE_BYTES;
-          // The leader announces the bytes of both CTAs' copies; the peer's copies may land first
-          // (the phase cannot complete before the leader's arrival).
-          if (leader) mbar_arrive_expect_tx(&full_bar[s], Cfg::STAGE_BYTES * (PAIR ? 2 : 1));
           const int k0 = kb * BK;
-          // A tiles: box {BK (k), 128 rows}.  B tiles: boxes {64 (n), BK (k rows)}.
-          load(st, &tmA0, k0, tm * kBM, &full_bar[s]);
-          uint8_t* bdst = st + Cfg::A_TILE;
-          if (NTERMS == 3) {
-            load(st + Cfg::A_TILE, &tmA1, k0, tm * kBM, &full_bar[s]);
-            bdst = st + 2 * Cfg::A_TILE;
-          }
+          if constexpr (FUSED) {
+            // A: one box {32 k (128 bytes), 128 rows}; B: boxes {32 columns (128 bytes), 32 k-rows}.
+            // Rows and columns outside the matrices arrive as zeros, and split(0) = (0, 0).
+            uint8_t* st = smem32 + s * Cfg::STAGE32_BYTES;
+            mbar_arrive_expect_tx(&ring_full[s], Cfg::STAGE32_BYTES);
+            load(st, &tmA0, k0, tm * kBM, &ring_full[s]);
 #pragma unroll
-          for (int a = 0; a < Cfg::BN_CTA / 64; ++a)
-            load(bdst + a * (BK * 128), &tmB0, n0 + a * 64, k0, &full_bar[s]);
-          if (NTERMS == 3) {
+            for (int a = 0; a < Cfg::BN_CTA / 32; ++a)
+              load(st + Cfg::A32_TILE + a * (BK * 128), &tmB0, n0 + a * 32, k0, &ring_full[s]);
+          } else {
+            uint8_t* st = smem + s * Cfg::STAGE_BYTES;
+            // The leader announces the bytes of both CTAs' copies; the peer's copies may land first
+            // (the phase cannot complete before the leader's arrival).
+            if (leader) mbar_arrive_expect_tx(&ring_full[s], Cfg::STAGE_BYTES * (PAIR ? 2 : 1));
+            // A tiles: box {BK (k), 128 rows}.  B tiles: boxes {64 (n), BK (k rows)}.
+            load(st, &tmA0, k0, tm * kBM, &ring_full[s]);
+            uint8_t* bdst = st + Cfg::A_TILE;
+            if (NTERMS == 3) {
+              load(st + Cfg::A_TILE, &tmA1, k0, tm * kBM, &ring_full[s]);
+              bdst = st + 2 * Cfg::A_TILE;
+            }
 #pragma unroll
             for (int a = 0; a < Cfg::BN_CTA / 64; ++a)
-              load(bdst + Cfg::B_TILE + a * (BK * 128), &tmB1, n0 + a * 64, k0, &full_bar[s]);
+              load(bdst + a * (BK * 128), &tmB0, n0 + a * 64, k0, &ring_full[s]);
+            if (NTERMS == 3) {
+#pragma unroll
+              for (int a = 0; a < Cfg::BN_CTA / 64; ++a)
+                load(bdst + Cfg::B_TILE + a * (BK * 128), &tmB1, n0 + a * 64, k0, &ring_full[s]);
+            }
           }
         }
       }
-      // Bounded drain: wait until the consumer has released every stage that was filled, so
-      // that no bulk copy is in flight when the CTA exits.
+      // No bulk copy may be in flight into this CTA's shared memory when it exits.  Normal end:
+      // wait until the consumer has released every stage that was filled.  After an abort the
+      // consumers no longer release anything: wait (bounded) for the copies themselves, on the
+      // barriers that count their bytes where this CTA can see them, else for a fixed time that
+      // is long against any copy's latency.
       if (ok) {
-        for (int d = 0; d < STAGES && d < (int)it; ++d, ++it) {
-          const int s = it % STAGES;
-          const uint32_t ph = (it / STAGES) & 1;
-          if (!mbar_wait_bounded(&empty_bar[s], ph ^ 1, abort_flag, p.err, kErrDrainWait)) break;
+        for (int d = 0; d < RING && d < (int)it; ++d, ++it) {
+          const int s = it % RING;
+          const uint32_t ph = (it / RING) & 1;
+          if (!mbar_wait_bounded(&ring_empty[s], ph ^ 1, abort_flag, p.err, kErrDrainWait, peer_abort)) {
+            ok = false;
+            break;
+          }
+        }
+      }
+      if (!ok) {
+        const uint32_t issued = it < (uint32_t)RING ? it : (uint32_t)RING;
+        if (FUSED || !PAIR || leader) {
+          for (uint32_t d = 1; d <= issued; ++d) {
+            const uint32_t j = it - d;
+            mbar_wait_clocks(&ring_full[j % RING], (j / RING) & 1, kAbortDrainClocks);
+          }
+        } else {
+          const long long t0 = clock64();
+          while (clock64() - t0 < kAbortDrainClocks) {}
         }
       }
     }
-  } else {
+  } else if (FUSED && warp >= kNumEpiWarps && warp < kNumEpiWarps + kNumConvWarps) {
     setmaxnreg_dec<88>();
-    // ------------------------------------------------------------------ converter warps (8-14)
-    // Per stage: A tile 128 x 32 FP32 = 512 items (ids 0-511: row m = id / 4, chunk q = id % 4 of
-    // 8 k), B tile 32 x 256 FP32 = 1024 items (ids 512-1535: k-row = (id - 512) / 32, chunk c of
-    // 8 n).  Thread t of the 224 takes ids t, t + 224, ..., t + 6 * 224 (the last round is partly
-    // idle).  A warp's 32 items are 8 rows x 128 bytes of A or one k-row x 1024 bytes of B:
-    // coalesced loads and bank-conflict-free 16-byte stores into the swizzled tiles.
-    //   A item -> byte offset m * 64 + ((q ^ ((m >> 1) & 3)) << 4) in the hi/lo A tile (64-byte swizzle)
-    //   B item -> atom (c / 8) * 4096 + k * 128 + (((c % 8) ^ (k % 8)) << 4) in the hi/lo B tile
-    // (PAIR: this CTA's B tile is 32 x 128, 512 items, ids 512-1023, 16 chunks per k-row.)
-    constexpr int kChunksPerRow = Cfg::BN_CTA / 8;                 // B chunks per k-row: 32 or 16
-    constexpr int kItems = 512 + BK * kChunksPerRow;               // 1536 or 1024
-    constexpr int kRounds = (kItems + kConvThreads - 1) / kConvThreads;   // 7 or 5
-    const int ct = threadIdx.x - kNumEpiWarps * 32;
-    const int lda = (int)p.lda32, ldb = (int)p.ldb32;
-    const bool wide_loads = ((lda | ldb) & 7) == 0 &&
-                            (((reinterpret_cast<uintptr_t>(p.A32) | reinterpret_cast<uintptr_t>(p.B32)) & 31) == 0);
-    // Geometry of item `id`, recomputed where it is used (keeping 14 offsets per thread alive next
-    // to 56 data registers costs more than these few integer operations).
-    auto smem_off = [&](int id) -> uint32_t {       // byte offset of the hi chunk inside the stage
-      if (id < 512) {
-        const int m = id >> 2, q = id & 3;
-        return (uint32_t)(m * 64 + ((q ^ ((m >> 1) & 3)) << 4));
-      }
-      const int b = id - 512, k = b / kChunksPerRow, c = b % kChunksPerRow;
-      return 2 * Cfg::A_TILE + (uint32_t)((c >> 3) * (BK * 128) + k * 128 + (((c & 7) ^ (k & 7)) << 4));
-    };
+    // ------------------------------------------------------------------ converter warps
+    // Per stage the FP32 ring holds A 128 x 32 (row m at m * 128 bytes, 16-byte chunk j of the row
+    // at position j ^ (m & 7): TMA's 128-byte swizzle) and B as BN_CTA / 32 boxes of 32 k-rows x
+    // 32 columns with the same row layout.  An item is 8 consecutive elements of a row (two
+    // chunks in, one hi chunk and one lo chunk out); a warp takes 32 items at a time:
+    //   A: 8 rows x 4 items.  Lane l: row l / 4, item l % 4.  A quarter warp reads 8 distinct
+    //      chunk positions (rows of both parities) and writes 128 contiguous bytes of the
+    //      64-byte-swizzled FP16 tile (row m at m * 64, chunk q at q ^ ((m >> 1) & 3)).
+    //   B: 2 k-rows (k even, k + 1) x 16 items, i.e. 128 columns.  Quarter warp w4, lanes 0-3:
+    //      row k, items 8 (w4 / 2) + 4 (w4 % 2) + 0..3; lanes 4-7: row k + 1, the other four items
+    //      of the same 64 columns.  Rows of both parities make the eight FP32 chunk positions
+    //      distinct, and the two groups of four land in complementary halves of a 128-byte row of
+    //      the FP16 atom (64 columns x 8 k-rows, chunk c at c ^ (k & 7)): no bank conflicts.
+    // Converter warp w takes A row blocks w, w + NW, ... and B row pairs w, w + NW, ... (both
+    // column halves when the CTA holds 256 columns), so (row & 7) and with it every swizzle term
+    // is a per-thread constant (NW a multiple of 4) and the rest of each address is an immediate.
+    constexpr int NW = kNumConvWarps;
+    static_assert(NW % 4 == 0 && 16 % NW == 0, "converter warps: 4, 8 or 16");
+    constexpr int RA = 16 / NW;                       // A rounds per stage
+    constexpr int RB = 16 / NW;                       // B row-pair rounds per stage
+    constexpr int HC = Cfg::BN_CTA / 128;             // column halves
+    const int cw = warp - kNumEpiWarps;
+    const int ar = lane >> 2, aq = lane & 3;
+    const uint32_t a_src_c = (uint32_t)(cw * 1024 + ar * 128 + (((2 * aq) ^ ar) << 4));
+    const uint32_t a_dst_c = (uint32_t)(cw * 512 + ar * 64 + ((aq ^ ((ar >> 1) & 3)) << 4));
+    const int w4 = lane >> 3, up = (lane >> 2) & 1, jj = lane & 3;
+    const int cl = 8 * (w4 >> 1) + 4 * ((w4 & 1) ^ up) + jj;      // item within the 128 columns
+    const int rowlow = ((2 * cw) & 7) | up;                       // (k-row & 7)
+    const uint32_t b_src_c = Cfg::A32_TILE +
+        (uint32_t)((cl >> 2) * (BK * 128) + (2 * cw + up) * 128 + (((2 * (cl & 3)) ^ rowlow) << 4));
+    const uint32_t b_dst_c = 2 * Cfg::A_TILE +
+        (uint32_t)((cl >> 3) * (BK * 128) + (2 * cw + up) * 128 + (((cl & 7) ^ rowlow) << 4));
     const int total_stages = (first_tile < num_tiles)
         ? ((num_tiles - first_tile + tile_stride - 1) / tile_stride) * num_kb : 0;
-    ConvItem item[kRounds];
-    // Coordinates of the stage whose FP32 data is being loaded (one stage ahead of conversion).
-    int ld_tile = first_tile, ld_kb = 0, ld_tm = 0, ld_tn = 0;
-    if (ld_tile < num_tiles) tile_rc(ld_tile, ld_tm, ld_tn);
-    auto load_round = [&](int r) {
-      const int id = ct + r * kConvThreads;
-      if (id >= kItems) return;
-      const int m0 = ld_tm * kBM, k0 = ld_kb * BK;
-      const int n0 = ld_tn * kBN + (PAIR ? (int)cta_rank * Cfg::BN_CTA : 0);
-      const bool interior = (m0 + kBM <= p.M) && (n0 + Cfg::BN_CTA <= p.N) && (k0 + BK <= p.K);
-      const bool is_a = id < 512;
-      const int row = is_a ? (id >> 2) : ((id - 512) / kChunksPerRow);     // tile row (A) / k-row (B)
-      const int col = is_a ? ((id & 3) * 8) : (((id - 512) % kChunksPerRow) * 8);
-      if (interior) {
-        const float* src = is_a ? (p.A32 + (long long)(m0 + row) * lda + (k0 + col))
-                                : (p.B32 + (long long)(k0 + row) * ldb + (n0 + col));
-        // volatile asm: the loads are issued here, one stage ahead of their use.  One 256-bit
-        // load per item when the rows are 32-byte aligned (a warp then reads 1 KB contiguously).
-        if (wide_loads) {
-          asm volatile("ld.global.nc.v8.f32 {%0, %1, %2, %3, %4, %5, %6, %7}, [%8];"
-                       : "=f"(item[r].a.x), "=f"(item[r].a.y), "=f"(item[r].a.z), "=f"(item[r].a.w),
-                         "=f"(item[r].b.x), "=f"(item[r].b.y), "=f"(item[r].b.z), "=f"(item[r].b.w)
-                       : "l"(src));
-        } else {
-          asm volatile("ld.global.nc.v4.f32 {%0, %1, %2, %3}, [%4];"
-                       : "=f"(item[r].a.x), "=f"(item[r].a.y), "=f"(item[r].a.z), "=f"(item[r].a.w)
-                       : "l"(src));
-          asm volatile("ld.global.nc.v4.f32 {%0, %1, %2, %3}, [%4 + 16];"
-                       : "=f"(item[r].b.x), "=f"(item[r].b.y), "=f"(item[r].b.z), "=f"(item[r].b.w)
-                       : "l"(src));
-        }
-      } else if (is_a) {
-        item[r] = load_item_guarded(p.A32, p.lda32, p.M, p.K, m0 + row, k0 + col);
-      } else {
-        item[r] = load_item_guarded(p.B32, p.ldb32, p.K, p.N, k0 + row, n0 + col);
-      }
-    };
-    if (total_stages > 0) {
-#pragma unroll
-      for (int r = 0; r < kRounds; ++r) load_round(r);
-    }
     ConvScale cs;
     cs.scale = p.scale;
     cs.fast = p.scale <= 32768.f;
     asm("mov.b64 %0, {%1, %1};" : "=l"(cs.scale2) : "f"(p.scale));
     cs.neg_scale_h = __half_as_ushort(__float2half_rn(cs.fast ? -p.scale : -1.f));
+    const uint32_t ring16 = smem_u32(smem), ring32 = smem_u32(smem32);
+    const bool timed = (blockIdx.x == 0 && threadIdx.x == kNumEpiWarps * 32);
+    (void)timed;
+    auto convert_stage = [&](uint32_t st32, uint32_t st16, auto fast_tag) {
+      constexpr bool FAST = decltype(fast_tag)::value;
+      const uint32_t a0 = st32 + a_src_c, a1 = a0 ^ 16u, ad = st16 + a_dst_c;
+#pragma unroll
+      for (int r = 0; r < RA; ++r)
+        convert_item<FAST>(a0 + r * NW * 1024, a1 + r * NW * 1024, ad + r * NW * 512, Cfg::A_TILE, cs);
+      const uint32_t b0 = st32 + b_src_c, b1 = b0 ^ 16u, bd = st16 + b_dst_c;
+#pragma unroll
+      for (int hc = 0; hc < HC; ++hc) {
+#pragma unroll
+        for (int r = 0; r < RB; ++r)
+          convert_item<FAST>(b0 + hc * 4 * (BK * 128) + r * NW * 256, b1 + hc * 4 * (BK * 128) + r * NW * 256,
+                             bd + hc * 2 * (BK * 128) + r * NW * 256, Cfg::B_TILE, cs);
+      }
+    };
     for (int it = 0; it < total_stages; ++it) {
       const int s = it % STAGES;
       const uint32_t ph = (it / STAGES) & 1;
-      // advance the load coordinates to stage it + 1
-      if (++ld_kb == num_kb) {
-        ld_kb = 0;
-        ld_tile += tile_stride;
-        if (ld_tile < num_tiles) tile_rc(ld_tile, ld_tm, ld_tn);
-      }
-      const bool more = (it + 1 < total_stages);
-      const bool timed = (blockIdx.x == 0 && ct == 0);
-      (void)timed;
       {
         SGC_T0();
-        if (!mbar_wait_bounded(&empty_bar[s], ph ^ 1, abort_flag, p.err, kErrConvEmptyWait)) break;
+        if (!mbar_wait_bounded(&full32_bar[s], ph, abort_flag, p.err, kErrConvFullWait, peer_abort)) break;
+        SGC_TADD(11, timed);
+      }
+      {
+        SGC_T0();
+        if (!mbar_wait_bounded(&empty_bar[s], ph ^ 1, abort_flag, p.err, kErrConvEmptyWait, peer_abort)) break;
         SGC_TADD(0, timed);
       }
       SGC_T0();
-      const uint32_t st = smem_u32(smem + s * Cfg::STAGE_BYTES);
-      // Convert the items loaded one stage ago; reload each register set as soon as it is free,
-      // so that about one stage of FP32 data per thread is always in flight.
-#pragma unroll
-      for (int r = 0; r < kRounds; ++r) {
-        const int id = ct + r * kConvThreads;
-        if (id < kItems) {
-          const uint32_t hi_addr = st + smem_off(id);
-          convert_store(item[r], cs, hi_addr, hi_addr + ((id < 512) ? Cfg::A_TILE : Cfg::B_TILE));
-          if (more) load_round(r);
-        }
-      }
+      const uint32_t st32 = ring32 + s * Cfg::STAGE32_BYTES, st16 = ring16 + s * Cfg::STAGE_BYTES;
+      if (cs.fast) convert_stage(st32, st16, std::true_type{});
+      else convert_stage(st32, st16, std::false_type{});
       SGC_TADD(1, timed);
       // Generic-proxy stores must be visible to the tensor core (async proxy) before the hand-over.
       {
@@ -921,6 +942,7 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA0, const __grid_constant__
         if (lane == 0) {
           if (!PAIR || leader) mbar_arrive(&full_bar[s]);
           else mbar_arrive_cluster(mapa_u32(smem_u32(&full_bar[s]), 0));   // the leader's barrier
+          mbar_arrive(&empty32_bar[s]);        // the FP32 stage may be refilled
         }
         SGC_TADD(2, timed);
       }
@@ -928,6 +950,10 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA0, const __grid_constant__
       if (timed) atomicAdd(&g_role_timing[3], 1ull);
 #endif
     }
+  } else {
+    // idle warps of the last warpgroup
+    if (FUSED) setmaxnreg_dec<88>();
+    else setmaxnreg_dec<56>();
   }
 
   // ---------------------------------------------------------------------- teardown

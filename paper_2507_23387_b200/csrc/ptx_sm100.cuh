@@ -58,25 +58,46 @@ __device__ __forceinline__ bool mbar_try_wait(uint64_t* bar, uint32_t parity) {
 // Wait limit in SM clocks (about 2 s at 1.9 GHz; the longest legitimate wait is one tile's
 // main loop, well under 10 ms).
 constexpr long long kWaitLimitClocks = 4000000000LL;
+// After an abort a producer waits this long (about 2 ms) for bulk copies that are still in flight.
+constexpr long long kAbortDrainClocks = 4000000LL;
+
+// Raise the abort flag of this CTA and, in a CTA pair, of the peer (its shared::cluster address;
+// 0 = no peer), so that every role of both CTAs leaves its wait loops promptly.
+__device__ __forceinline__ void raise_abort(volatile uint32_t* abort_flag, uint32_t peer_abort_addr) {
+  if (abort_flag != nullptr) *abort_flag = 1u;
+  if (peer_abort_addr != 0u)
+    asm volatile("st.shared::cluster.u32 [%0], %1;" ::"r"(peer_abort_addr), "r"(1u) : "memory");
+}
 
 // Bounded wait.  Returns false if the CTA is aborting or the limit ran out; in the latter case
 // the first failing waiter publishes `code` in the global error word and raises the abort flag.
 // With abort_flag == nullptr only the clock limit ends the wait (used when draining at exit).
 __device__ __forceinline__ bool mbar_wait_bounded(uint64_t* bar, uint32_t parity,
                                                   volatile uint32_t* abort_flag,
-                                                  unsigned int* err_word, unsigned int code) {
+                                                  unsigned int* err_word, unsigned int code,
+                                                  uint32_t peer_abort_addr = 0u,
+                                                  long long limit = kWaitLimitClocks) {
   if (mbar_try_wait(bar, parity)) return true;
   const long long t0 = clock64();
   while (true) {
     if (mbar_try_wait(bar, parity)) return true;
     if (abort_flag != nullptr && *abort_flag) return false;
-    if (clock64() - t0 > kWaitLimitClocks) {
-      if (abort_flag != nullptr) *abort_flag = 1u;
+    if (clock64() - t0 > limit) {
+      raise_abort(abort_flag, peer_abort_addr);
       atomicCAS(err_word, 0u, code);
       __threadfence();
       return false;
     }
   }
+}
+
+// Plain bounded wait without side effects: true if the phase completed within `limit` clocks.
+__device__ __forceinline__ bool mbar_wait_clocks(uint64_t* bar, uint32_t parity, long long limit) {
+  const long long t0 = clock64();
+  while (!mbar_try_wait(bar, parity)) {
+    if (clock64() - t0 > limit) return false;
+  }
+  return true;
 }
 
 // ----------------------------------------------------------------------------- fences
@@ -249,14 +270,16 @@ __device__ __forceinline__ bool mbar_try_wait_cluster(uint64_t* bar, uint32_t pa
 // Bounded wait with cluster-scope acquire (the arrivals may come from the peer CTA).
 __device__ __forceinline__ bool mbar_wait_bounded_cluster(uint64_t* bar, uint32_t parity,
                                                           volatile uint32_t* abort_flag,
-                                                          unsigned int* err_word, unsigned int code) {
+                                                          unsigned int* err_word, unsigned int code,
+                                                          uint32_t peer_abort_addr = 0u,
+                                                          long long limit = kWaitLimitClocks) {
   if (mbar_try_wait_cluster(bar, parity)) return true;
   const long long t0 = clock64();
   while (true) {
     if (mbar_try_wait_cluster(bar, parity)) return true;
     if (abort_flag != nullptr && *abort_flag) return false;
-    if (clock64() - t0 > kWaitLimitClocks) {
-      if (abort_flag != nullptr) *abort_flag = 1u;
+    if (clock64() - t0 > limit) {
+      raise_abort(abort_flag, peer_abort_addr);
       atomicCAS(err_word, 0u, code);
       __threadfence();
       return false;

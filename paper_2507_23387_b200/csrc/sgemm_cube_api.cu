@@ -127,8 +127,9 @@ int set_kernel_attrs(sgemm_cube_ctx* h) {
 // only uses them when asked to.
 bool use_pair(const sgemm_cube_ctx* h, int M, int N, bool fused) {
   (void)N;
+  (void)fused;
   if (h->cta_pair != 2) return h->cta_pair == 1;
-  return !fused && M > sgc::kBM;
+  return M > sgc::kBM;
 }
 
 // Launch one tensor-core kernel: a persistent grid of single CTAs, or of 2-CTA clusters (PAIR).
@@ -382,10 +383,22 @@ int launch_fused(sgemm_cube_ctx* h, int M, int N, int K, const float* A, int64_t
   p.B32 = B; p.ldb32 = ldb;
   p.scale = ldexpf(1.0f, s);
   p.ksplit = 1; p.kslice_blocks = 0; p.Phh = nullptr; p.Px = nullptr; p.pstride = 0; p.ldp = 0;
-  CUtensorMap unused;
-  memset(&unused, 0, sizeof(unused));
-  return use_pair(h, M, N, true) ? launch_tc_kernel<3, true, true>(h, M, N, unused, unused, unused, unused, p, st)
-                           : launch_tc_kernel<3, true, false>(h, M, N, unused, unused, unused, unused, p, st);
+  // FP32 tiles as TMA stages them for the converter warps: A in boxes of {BK k, 128 rows}, B in
+  // boxes of {32 columns, BK k-rows}, both with the 128-byte swizzle (rows of 128 bytes).
+  CUtensorMap tmA, tmB;
+  rc = make_map(h, &tmA, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 4, A, K, M, lda, Cfg::BK, sgc::kBM,
+                CU_TENSOR_MAP_SWIZZLE_128B);
+  if (rc) return rc;
+  rc = make_map(h, &tmB, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 4, B, N, K, ldb, 32, Cfg::BK,
+                CU_TENSOR_MAP_SWIZZLE_128B);
+  if (rc) return rc;
+  if (use_pair(h, M, N, true)) {
+    rc = launch_tc_kernel<3, true, true>(h, M, N, tmA, tmA, tmB, tmB, p, st);
+    // Clusters that cannot be scheduled: when the pair mode was the library's own choice, single
+    // CTAs compute the same bits.
+    if (rc != SGEMM_CUBE_CUDA_ERROR || h->cta_pair != 2) return rc;
+  }
+  return launch_tc_kernel<3, true, false>(h, M, N, tmA, tmA, tmB, tmB, p, st);
 }
 
 // sgemm_cube, strategy "two-phase": split both operands once into the handle's workspace, then one

@@ -51,8 +51,8 @@ constexpr int kTcThreads = 384;     // not FUSED: + TMA warp + MMA warp (+ 2 idl
 #define SGC_CONV_WARPS 4
 #endif
 constexpr int kNumConvWarps = SGC_CONV_WARPS;      // a multiple of 4 (see the converter role)
-// FUSED: + converter warps + MMA warp + TMA warp, rounded up to whole warpgroups
-constexpr int kFusedThreads = ((kNumEpiWarps + kNumConvWarps + 2 + 3) / 4) * 128;
+// FUSED: + converter warps + MMA warp + TMA warp + 2 relay warps, rounded up to whole warpgroups
+constexpr int kFusedThreads = ((kNumEpiWarps + kNumConvWarps + 4 + 3) / 4) * 128;
 constexpr uint32_t kTmemCols = 512;
 
 // error codes written to the device error word (which wait gave up)
@@ -64,6 +64,7 @@ enum : unsigned int {
   kErrDrainWait = 0x105,
   kErrConvEmptyWait = 0x106,
   kErrConvFullWait = 0x107,
+  kErrRelayWait = 0x108,
 };
 
 // Optional role timing (compile with -DSGC_ROLE_TIMING): CTA 0 adds the clocks each role spends in
@@ -229,29 +230,34 @@ __device__ __forceinline__ void split_pair_fast(uint64_t xp, uint64_t scale2, ui
 }
 
 // One item: FP32 chunks at shared addresses src0 / src1 (elements 0-3 / 4-7) -> hi chunk at dst,
-// lo chunk at dst + lo_off.
+// lo chunk at dst + lo_off.  Loading and converting are separate so that a warp can have the
+// loads of several items in flight before it starts on the arithmetic of the first.
+struct ConvItem { uint64_t x01, x23, x45, x67; };
+
+__device__ __forceinline__ void load_item(ConvItem& it, uint32_t src0, uint32_t src1) {
+  asm volatile("ld.shared.v2.b64 {%0, %1}, [%2];" : "=l"(it.x01), "=l"(it.x23) : "r"(src0));
+  asm volatile("ld.shared.v2.b64 {%0, %1}, [%2];" : "=l"(it.x45), "=l"(it.x67) : "r"(src1));
+}
+
 template <bool FAST>
-__device__ __forceinline__ void convert_item(uint32_t src0, uint32_t src1, uint32_t dst, uint32_t lo_off,
-                                             const ConvScale& cs) {
-  uint64_t x01, x23, x45, x67;
-  asm volatile("ld.shared.v2.b64 {%0, %1}, [%2];" : "=l"(x01), "=l"(x23) : "r"(src0) : "memory");
-  asm volatile("ld.shared.v2.b64 {%0, %1}, [%2];" : "=l"(x45), "=l"(x67) : "r"(src1) : "memory");
+__device__ __forceinline__ void convert_store(const ConvItem& it, uint32_t dst, uint32_t lo_off,
+                                              const ConvScale& cs) {
   uint4 h, l;
   if (FAST) {
-    split_pair_fast(x01, cs.scale2, cs.neg_scale_h, h.x, l.x);
-    split_pair_fast(x23, cs.scale2, cs.neg_scale_h, h.y, l.y);
-    split_pair_fast(x45, cs.scale2, cs.neg_scale_h, h.z, l.z);
-    split_pair_fast(x67, cs.scale2, cs.neg_scale_h, h.w, l.w);
+    split_pair_fast(it.x01, cs.scale2, cs.neg_scale_h, h.x, l.x);
+    split_pair_fast(it.x23, cs.scale2, cs.neg_scale_h, h.y, l.y);
+    split_pair_fast(it.x45, cs.scale2, cs.neg_scale_h, h.z, l.z);
+    split_pair_fast(it.x67, cs.scale2, cs.neg_scale_h, h.w, l.w);
   } else {
-    split_pair(x01, cs.scale, h.x, l.x);
-    split_pair(x23, cs.scale, h.y, l.y);
-    split_pair(x45, cs.scale, h.z, l.z);
-    split_pair(x67, cs.scale, h.w, l.w);
+    split_pair(it.x01, cs.scale, h.x, l.x);
+    split_pair(it.x23, cs.scale, h.y, l.y);
+    split_pair(it.x45, cs.scale, h.z, l.z);
+    split_pair(it.x67, cs.scale, h.w, l.w);
   }
   asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(dst), "r"(h.x), "r"(h.y),
-               "r"(h.z), "r"(h.w) : "memory");
+               "r"(h.z), "r"(h.w));
   asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(dst + lo_off), "r"(l.x), "r"(l.y),
-               "r"(l.z), "r"(l.w) : "memory");
+               "r"(l.z), "r"(l.w));
 }
 
 __device__ __forceinline__ void tmem_ld_cols(uint32_t taddr, uint32_t (&r)[16]) { tmem_ld_32x32b_x16(taddr, r); }
@@ -296,12 +302,13 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA0, const __grid_constant__
   uint64_t* drain_bar = bars + 2 * STAGES + 4;   // [1]
   uint64_t* full32_bar = bars + 2 * STAGES + 5;              // [STAGES32]  TMA -> converters
   uint64_t* empty32_bar = bars + 2 * STAGES + 5 + STAGES32;  // [STAGES32]  converters -> TMA
-  uint32_t* tmem_base_slot = reinterpret_cast<uint32_t*>(bars + 2 * STAGES + 5 + 2 * STAGES32);
+  uint64_t* conv_bar = bars + 2 * STAGES + 5 + 2 * STAGES32;   // [STAGES32]  converters -> relay thread
+  uint32_t* tmem_base_slot = reinterpret_cast<uint32_t*>(bars + 2 * STAGES + 5 + 3 * STAGES32);
   volatile uint32_t* abort_flag = tmem_base_slot + 1;
   // PAIR: a wait that gives up also raises the peer's flag (shared::cluster address of the same slot)
   const uint32_t peer_abort =
       PAIR ? mapa_u32(smem_u32(tmem_base_slot + 1), cta_rank ^ 1u) : 0u;
-  static_assert((2 * STAGES + 5 + 2 * STAGES32) * 8 + 8 <= 256, "barrier block");
+  static_assert((2 * STAGES + 5 + 3 * STAGES32) * 8 + 8 <= 256, "barrier block");
   uint8_t* store_staging = smem + Cfg::RING_BYTES + 256;   // epilogue transposition buffers
 
   const int warp = threadIdx.x >> 5;
@@ -317,7 +324,7 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA0, const __grid_constant__
 
   if (threadIdx.x == 0) {
     for (int s = 0; s < STAGES; ++s) {
-      mbar_init(&full_bar[s], FUSED ? kNumConvWarps * (PAIR ? 2 : 1) : 1);
+      mbar_init(&full_bar[s], (FUSED && PAIR) ? 2 : 1);   // FUSED: one relay thread per CTA
       mbar_init(&empty_bar[s], 1);
     }
     for (int r = 0; r < 2; ++r) {
@@ -327,6 +334,7 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA0, const __grid_constant__
     for (int s = 0; s < STAGES32; ++s) {
       mbar_init(&full32_bar[s], 1);
       mbar_init(&empty32_bar[s], kNumConvWarps);
+      mbar_init(&conv_bar[s], kNumConvWarps);
     }
     mbar_init(drain_bar, 1);
     *abort_flag = 0u;
@@ -407,7 +415,6 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA0, const __grid_constant__
           SGC_T0();
           if (!wait_tfull(r_main)) { ok = false; break; }
           SGC_TADD(6, blockIdx.x == 0 && threadIdx.x == 0);
-          SGC_TADD(13, blockIdx.x == 1 && threadIdx.x == 0);
         }
         SGC_T0();
         tc_fence_after_sync();
@@ -481,7 +488,6 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA0, const __grid_constant__
         }
         }  // not reordered
         SGC_TADD(7, blockIdx.x == 0 && threadIdx.x == 0);
-        SGC_TADD(14, blockIdx.x == 1 && threadIdx.x == 0);
       }
       if (!ok) break;
       SGC_T0();
@@ -791,9 +797,13 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA0, const __grid_constant__
         for (int kb = kb0; kb < kb1; ++kb, ++it) {
           const int s = it % RING;
           const uint32_t ph = (it / RING) & 1;
-          if (!mbar_wait_bounded(&ring_empty[s], ph ^ 1, abort_flag, p.err, kErrProducerEmptyWait, peer_abort)) {
-            ok = false;
-            break;
+          {
+            SGC_T0();
+            if (!mbar_wait_bounded(&ring_empty[s], ph ^ 1, abort_flag, p.err, kErrProducerEmptyWait, peer_abort)) {
+              ok = false;
+              break;
+            }
+            SGC_TADD(14, blockIdx.x == 0);
           }
           const int k0 = kb * BK;
           if constexpr (FUSED) {
@@ -899,20 +909,29 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA0, const __grid_constant__
     cs.neg_scale_h = __half_as_ushort(__float2half_rn(cs.fast ? -p.scale : -1.f));
     const uint32_t ring16 = smem_u32(smem), ring32 = smem_u32(smem32);
     const bool timed = (blockIdx.x == 0 && threadIdx.x == kNumEpiWarps * 32);
-    (void)timed;
+    const bool timed1 = (blockIdx.x == 1 && threadIdx.x == (kNumEpiWarps + kNumConvWarps - 1) * 32);
+    (void)timed; (void)timed1;
     auto convert_stage = [&](uint32_t st32, uint32_t st16, auto fast_tag) {
       constexpr bool FAST = decltype(fast_tag)::value;
+      // batches of RA (= RB) items: all loads of a batch are issued before its arithmetic
       const uint32_t a0 = st32 + a_src_c, a1 = a0 ^ 16u, ad = st16 + a_dst_c;
+      {
+        ConvItem x[RA];
 #pragma unroll
-      for (int r = 0; r < RA; ++r)
-        convert_item<FAST>(a0 + r * NW * 1024, a1 + r * NW * 1024, ad + r * NW * 512, Cfg::A_TILE, cs);
+        for (int r = 0; r < RA; ++r) load_item(x[r], a0 + r * NW * 1024, a1 + r * NW * 1024);
+#pragma unroll
+        for (int r = 0; r < RA; ++r) convert_store<FAST>(x[r], ad + r * NW * 512, Cfg::A_TILE, cs);
+      }
       const uint32_t b0 = st32 + b_src_c, b1 = b0 ^ 16u, bd = st16 + b_dst_c;
 #pragma unroll
       for (int hc = 0; hc < HC; ++hc) {
+        ConvItem x[RB];
 #pragma unroll
         for (int r = 0; r < RB; ++r)
-          convert_item<FAST>(b0 + hc * 4 * (BK * 128) + r * NW * 256, b1 + hc * 4 * (BK * 128) + r * NW * 256,
-                             bd + hc * 2 * (BK * 128) + r * NW * 256, Cfg::B_TILE, cs);
+          load_item(x[r], b0 + hc * 4 * (BK * 128) + r * NW * 256, b1 + hc * 4 * (BK * 128) + r * NW * 256);
+#pragma unroll
+        for (int r = 0; r < RB; ++r)
+          convert_store<FAST>(x[r], bd + hc * 2 * (BK * 128) + r * NW * 256, Cfg::B_TILE, cs);
       }
     };
     for (int it = 0; it < total_stages; ++it) {
@@ -933,27 +952,51 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA0, const __grid_constant__
       if (cs.fast) convert_stage(st32, st16, std::true_type{});
       else convert_stage(st32, st16, std::false_type{});
       SGC_TADD(1, timed);
-      // Generic-proxy stores must be visible to the tensor core (async proxy) before the hand-over.
+      // Hand the stage to the relay thread (which makes it visible to the tensor core) and the
+      // FP32 stage back to the TMA producer.
       {
         SGC_T0();
-        if (PAIR) fence_proxy_async_smem_cluster();
-        else fence_proxy_async_smem();
         __syncwarp();
         if (lane == 0) {
-          if (!PAIR || leader) mbar_arrive(&full_bar[s]);
-          else mbar_arrive_cluster(mapa_u32(smem_u32(&full_bar[s]), 0));   // the leader's barrier
-          mbar_arrive(&empty32_bar[s]);        // the FP32 stage may be refilled
+          mbar_arrive(&conv_bar[s]);
+          mbar_arrive(&empty32_bar[s]);
         }
         SGC_TADD(2, timed);
+        SGC_TADD(15, timed1);
       }
 #ifdef SGC_ROLE_TIMING
       if (timed) atomicAdd(&g_role_timing[3], 1ull);
 #endif
     }
+  } else if (FUSED) {
+    setmaxnreg_dec<88>();
+    // ------------------------------------------------------------------ relay threads
+    // The converters' stores go through the generic proxy and the tensor core reads through the
+    // async proxy, so a proxy fence has to lie between the two.  Inside a cluster that fence
+    // costs several hundred clocks (and the peer's arrival on the leader's barrier as much
+    // again), which the converter warps cannot afford once per stage.  The fence may be executed
+    // by any thread on the path from the stores to the MMA: the converter warps arrive on a
+    // local barrier, one lane of each of the two spare warps takes every other stage, acquires
+    // that barrier, fences and tells the MMA thread (in a pair: the leader's) that this CTA's
+    // part of the stage is ready.
+    const int rw = warp - (kProducerWarp + 1);         // 0 or 1
+    if (lane == 0 && rw >= 0 && rw < 2) {
+      const int total_stages = (first_tile < num_tiles)
+          ? ((num_tiles - first_tile + tile_stride - 1) / tile_stride) * num_kb : 0;
+      for (int it = rw; it < total_stages; it += 2) {
+        const int s = it % STAGES;
+        const uint32_t ph = (it / STAGES) & 1;
+        if (!mbar_wait_bounded(&conv_bar[s], ph, abort_flag, p.err, kErrRelayWait, peer_abort)) break;
+        SGC_T0();
+        fence_proxy_async_smem();
+        if (!PAIR || leader) mbar_arrive(&full_bar[s]);
+        else mbar_arrive_cluster(mapa_u32(smem_u32(&full_bar[s]), 0));   // the leader's barrier
+        SGC_TADD(12, blockIdx.x == 1 && rw == 0);
+        SGC_TADD(13, blockIdx.x == 0 && rw == 0);
+      }
+    }
   } else {
-    // idle warps of the last warpgroup
-    if (FUSED) setmaxnreg_dec<88>();
-    else setmaxnreg_dec<56>();
+    setmaxnreg_dec<56>();      // idle warps of the last warpgroup
   }
 
   // ---------------------------------------------------------------------- teardown

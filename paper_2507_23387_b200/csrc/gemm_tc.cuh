@@ -47,6 +47,12 @@ constexpr int kBM = 128;            // CTA tile rows  (UMMA M)
 constexpr int kBN = 256;            // CTA tile cols  (UMMA N)
 constexpr int kNumEpiWarps = 8;     // warps 0-7
 constexpr int kTcThreads = 384;     // not FUSED: + TMA warp + MMA warp (+ 2 idle warps: whole warpgroup)
+#ifndef SGC_RELAY_ARRIVE
+#define SGC_RELAY_ARRIVE 1
+#endif
+#ifndef SGC_L2_PREFETCH
+#define SGC_L2_PREFETCH 0
+#endif
 #ifndef SGC_CONV_WARPS
 #define SGC_CONV_WARPS 4
 #endif
@@ -815,6 +821,14 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA0, const __grid_constant__
 #pragma unroll
             for (int a = 0; a < Cfg::BN_CTA / 32; ++a)
               load(st + Cfg::A32_TILE + a * (BK * 128), &tmB0, n0 + a * 32, k0, &ring_full[s]);
+#if SGC_L2_PREFETCH > 0
+            if (kb + SGC_L2_PREFETCH < kb1) {
+              const int kp = k0 + SGC_L2_PREFETCH * BK;
+              tma_prefetch_l2_2d(&tmA0, kp, tm * kBM);
+#pragma unroll
+              for (int a = 0; a < Cfg::BN_CTA / 32; ++a) tma_prefetch_l2_2d(&tmB0, n0 + a * 32, kp);
+            }
+#endif
           } else {
             uint8_t* st = smem + s * Cfg::STAGE_BYTES;
             // The leader announces the bytes of both CTAs' copies; the peer's copies may land first
@@ -990,7 +1004,13 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA0, const __grid_constant__
         SGC_T0();
         fence_proxy_async_smem();
         if (!PAIR || leader) mbar_arrive(&full_bar[s]);
+#if SGC_RELAY_ARRIVE == 0
         else mbar_arrive_cluster(mapa_u32(smem_u32(&full_bar[s]), 0));   // the leader's barrier
+#elif SGC_RELAY_ARRIVE == 1
+        else mbar_arrive_remote_cta(mapa_u32(smem_u32(&full_bar[s]), 0));
+#else
+        else mbar_arrive_cluster_relaxed(mapa_u32(smem_u32(&full_bar[s]), 0));
+#endif
         SGC_TADD(12, blockIdx.x == 1 && rw == 0);
         SGC_TADD(13, blockIdx.x == 0 && rw == 0);
       }

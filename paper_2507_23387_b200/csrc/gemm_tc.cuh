@@ -50,9 +50,6 @@ constexpr int kTcThreads = 384;     // not FUSED: + TMA warp + MMA warp (+ 2 idl
 #ifndef SGC_RELAY_ARRIVE
 #define SGC_RELAY_ARRIVE 1
 #endif
-#ifndef SGC_L2_PREFETCH
-#define SGC_L2_PREFETCH 0
-#endif
 #ifndef SGC_CONV_WARPS
 #define SGC_CONV_WARPS 4
 #endif
@@ -129,16 +126,25 @@ struct TcCfg {
   static constexpr int A_ROW_BYTES = BK * 2;              // 128 or 64: also the swizzle span of A
   static constexpr uint32_t A_TILE = kBM * BK * 2;        // one FP16 A tile
   static constexpr uint32_t B_TILE = BK * BN_CTA * 2;     // one FP16 B tile (this CTA's columns)
-  static constexpr uint32_t STAGE_BYTES = (NTERMS == 1) ? (A_TILE + B_TILE) : 2 * (A_TILE + B_TILE);
-  // FUSED: a second ring holds the FP32 tiles that TMA stages for the converter warps (same k
-  // depth, same bytes per stage as the (hi, lo) pair it becomes); the two rings share the space.
+  // FUSED: a stage is filled by TMA with the FP32 tiles (A: 128 rows x BK; B: BN_CTA / 32 boxes of
+  // BK k-rows x 32 columns; rows of 128 bytes, 128-byte swizzle) and converted IN PLACE: every
+  // 1 KB region (8 rows x 32 FP32 elements) becomes the 512-byte hi atom and the 512-byte lo atom
+  // of the same 8 x 32 elements (rows of 64 bytes, 64-byte swizzle).  One ring, each slot going
+  // TMA -> converters -> MMA -> TMA, so the same bytes hold a tile in flight, a tile being split
+  // and a tile being multiplied, whichever the pipeline needs more of.
   static constexpr uint32_t A32_TILE = FUSED ? kBM * BK * 4 : 0;
-  static constexpr uint32_t B32_TILE = FUSED ? BK * BN_CTA * 4 : 0;   // BN_CTA / 32 boxes of 32 columns
-  static constexpr uint32_t STAGE32_BYTES = A32_TILE + B32_TILE;
-  static constexpr int STAGES = FUSED ? (int)(196608 / (STAGE_BYTES + STAGE32_BYTES))
-                                      : ((196608 / STAGE_BYTES) > 8 ? 8 : (int)(196608 / STAGE_BYTES));
-  static constexpr int STAGES32 = FUSED ? STAGES : 0;
-  static constexpr uint32_t RING_BYTES = STAGES * STAGE_BYTES + STAGES32 * STAGE32_BYTES;
+  static constexpr uint32_t B32_TILE = FUSED ? BK * BN_CTA * 4 : 0;
+  static constexpr uint32_t STAGE_BYTES =
+      FUSED ? (A32_TILE + B32_TILE) : ((NTERMS == 1) ? (A_TILE + B_TILE) : 2 * (A_TILE + B_TILE));
+  static constexpr int STAGES = (196608 / STAGE_BYTES) > 8 ? 8 : (int)(196608 / STAGE_BYTES);
+  static constexpr uint32_t RING_BYTES = STAGES * STAGE_BYTES;
+  // Where the MMA thread finds the operands of a stage, and their descriptor strides.
+  static constexpr uint32_t A_LO_OFF = FUSED ? 512 : A_TILE;                 // lo_A relative to hi_A
+  static constexpr uint32_t B_OFF = FUSED ? A32_TILE : ((NTERMS == 3) ? 2 * A_TILE : A_TILE);
+  static constexpr uint32_t B_LO_OFF = FUSED ? 512 : B_TILE;                 // lo_B relative to hi_B
+  static constexpr uint32_t A_SBO = FUSED ? 1024 : 8 * A_ROW_BYTES;          // next 8 rows of A
+  static constexpr uint32_t B_LBO = BK * 128;    // next column atom of B (64 columns; FUSED: 32)
+  static constexpr uint32_t B_SBO = 1024;        // next 8 k-rows of the same columns
   static constexpr uint32_t STORE_STAGING = kNumEpiWarps * 4096;   // 32 rows x 128 bytes per warp
   static constexpr uint32_t SMEM_BYTES =
       RING_BYTES + 1024 /*align*/ + 256 /*barriers*/ + STORE_STAGING;
@@ -291,7 +297,6 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA0, const __grid_constant__
   // not FUSED: warp 8 loads FP16 tiles; FUSED: the warp after the MMA warp loads FP32 tiles
   constexpr int kMmaWarp = FUSED ? kNumEpiWarps + kNumConvWarps : 9;
   constexpr int kProducerWarp = FUSED ? kMmaWarp + 1 : 8;
-  constexpr int STAGES32 = Cfg::STAGES32;
   static_assert(!FUSED || NTERMS == 3, "the fused kernel computes all three products");
 
   extern __shared__ uint8_t smem_raw[];
@@ -299,22 +304,21 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA0, const __grid_constant__
   // of the shared-memory address bits, so every tile must start on a 1024-byte boundary.
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) &
                                              ~uintptr_t(1023));
-  uint8_t* smem32 = smem + STAGES * Cfg::STAGE_BYTES;       // FUSED: the FP32 ring
   uint64_t* bars = reinterpret_cast<uint64_t*>(smem + Cfg::RING_BYTES);
-  uint64_t* full_bar = bars;                 // [STAGES]  producer/converters -> MMA
-  uint64_t* empty_bar = bars + STAGES;       // [STAGES]  MMA -> producer/converters
+  uint64_t* full_bar = bars;                 // [STAGES]  producer (FUSED: relay threads) -> MMA
+  uint64_t* empty_bar = bars + STAGES;       // [STAGES]  MMA -> producer
   uint64_t* tfull_bar = bars + 2 * STAGES;   // [2]       MMA -> epilogue (TMEM region filled)
   uint64_t* tempty_bar = bars + 2 * STAGES + 2;  // [2]   epilogue -> MMA (TMEM region drained)
   uint64_t* drain_bar = bars + 2 * STAGES + 4;   // [1]
-  uint64_t* full32_bar = bars + 2 * STAGES + 5;              // [STAGES32]  TMA -> converters
-  uint64_t* empty32_bar = bars + 2 * STAGES + 5 + STAGES32;  // [STAGES32]  converters -> TMA
-  uint64_t* conv_bar = bars + 2 * STAGES + 5 + 2 * STAGES32;   // [STAGES32]  converters -> relay thread
-  uint32_t* tmem_base_slot = reinterpret_cast<uint32_t*>(bars + 2 * STAGES + 5 + 3 * STAGES32);
+  constexpr int kFusedBars = FUSED ? STAGES : 0;
+  uint64_t* full32_bar = bars + 2 * STAGES + 5;              // [STAGES]  FUSED: TMA -> converters
+  uint64_t* conv_bar = bars + 2 * STAGES + 5 + kFusedBars;   // [STAGES]  FUSED: converters -> relay
+  uint32_t* tmem_base_slot = reinterpret_cast<uint32_t*>(bars + 2 * STAGES + 5 + 2 * kFusedBars);
   volatile uint32_t* abort_flag = tmem_base_slot + 1;
   // PAIR: a wait that gives up also raises the peer's flag (shared::cluster address of the same slot)
   const uint32_t peer_abort =
       PAIR ? mapa_u32(smem_u32(tmem_base_slot + 1), cta_rank ^ 1u) : 0u;
-  static_assert((2 * STAGES + 5 + 3 * STAGES32) * 8 + 8 <= 256, "barrier block");
+  static_assert((2 * STAGES + 5 + 2 * kFusedBars) * 8 + 8 <= 256, "barrier block");
   uint8_t* store_staging = smem + Cfg::RING_BYTES + 256;   // epilogue transposition buffers
 
   const int warp = threadIdx.x >> 5;
@@ -337,9 +341,8 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA0, const __grid_constant__
       mbar_init(&tfull_bar[r], 1);
       mbar_init(&tempty_bar[r], kNumEpiWarps * (PAIR ? 2 : 1));
     }
-    for (int s = 0; s < STAGES32; ++s) {
+    for (int s = 0; s < kFusedBars; ++s) {
       mbar_init(&full32_bar[s], 1);
-      mbar_init(&empty32_bar[s], kNumConvWarps);
       mbar_init(&conv_bar[s], kNumConvWarps);
     }
     mbar_init(drain_bar, 1);
@@ -607,9 +610,8 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA0, const __grid_constant__
       };
       constexpr uint64_t a_swz = (Cfg::A_ROW_BYTES == 128) ? kSwizzle128
                                  : (Cfg::A_ROW_BYTES == 64) ? kSwizzle64 : kSwizzle32;
-      constexpr uint32_t a_sbo = 8 * Cfg::A_ROW_BYTES;     // 8 rows of the swizzle atom
-      constexpr uint32_t b_lbo = BK * 128;                 // next 64-column atom of B
-      constexpr uint32_t b_sbo = 1024;                     // next 8 k-rows inside an atom
+      constexpr uint64_t b_swz = FUSED ? kSwizzle64 : kSwizzle128;
+      constexpr uint32_t a_sbo = Cfg::A_SBO, b_lbo = Cfg::B_LBO, b_sbo = Cfg::B_SBO;
       // The issuing thread is a single lane: every instruction it spends on a descriptor delays
       // the next MMA.  Only the start-address field (low word, in units of 16 bytes) changes from
       // one MMA to the next, so the constant fields are folded at compile time and a descriptor
@@ -617,7 +619,7 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA0, const __grid_constant__
       constexpr uint32_t a_desc_hi =
           ((a_sbo >> 4) & 0x3FFFu) | (1u << 14) | ((uint32_t)a_swz << 29);
       constexpr uint32_t b_desc_hi =
-          ((b_sbo >> 4) & 0x3FFFu) | (1u << 14) | ((uint32_t)kSwizzle128 << 29);
+          ((b_sbo >> 4) & 0x3FFFu) | (1u << 14) | ((uint32_t)b_swz << 29);
       constexpr uint32_t a_desc_lo0 = ((16u >> 4) & 0x3FFFu) << 16;
       constexpr uint32_t b_desc_lo0 = ((b_lbo >> 4) & 0x3FFFu) << 16;
       auto desc = [](uint32_t lo, uint32_t hi) -> uint64_t {
@@ -659,9 +661,9 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA0, const __grid_constant__
               tc_fence_after_sync();
               x_ready = true;
             }
-            const uint32_t a_hi = a_desc_lo0 + (st >> 4), a_lo = a_hi + (Cfg::A_TILE >> 4);
-            const uint32_t b_hi = b_desc_lo0 + ((st + 2 * Cfg::A_TILE) >> 4);
-            const uint32_t b_lo = b_hi + (Cfg::B_TILE >> 4);
+            const uint32_t a_hi = a_desc_lo0 + (st >> 4), a_lo = a_hi + (Cfg::A_LO_OFF >> 4);
+            const uint32_t b_hi = b_desc_lo0 + ((st + Cfg::B_OFF) >> 4);
+            const uint32_t b_lo = b_hi + (Cfg::B_LO_OFF >> 4);
             // Order inside the correction chain: per 32 k-steps, lo*hi of both k16 steps, then
             // hi*lo of both.  Fixed whatever the stage depth, so that every variant of the
             // kernel rounds the chain identically.
@@ -693,7 +695,7 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA0, const __grid_constant__
               main_ready = true;
             }
             const uint32_t a_hi = a_desc_lo0 + (st >> 4);
-            const uint32_t b_hi = b_desc_lo0 + ((st + ((NTERMS == 3) ? 2 * Cfg::A_TILE : Cfg::A_TILE)) >> 4);
+            const uint32_t b_hi = b_desc_lo0 + ((st + Cfg::B_OFF) >> 4);
 #pragma unroll
             for (int j = 0; j < BK / 16; ++j) {
               const uint64_t da = desc(a_hi + 2 * j, a_desc_hi);
@@ -783,13 +785,14 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA0, const __grid_constant__
     if (FUSED) setmaxnreg_dec<88>();
     else setmaxnreg_dec<56>();
     // ------------------------------------------------------------------ TMA producer
-    // not FUSED: FP16 operand tiles into the ring the MMA thread reads.  FUSED: FP32 tiles of A
-    // and B into the FP32 ring the converter warps read (this CTA's own rows of A and its own
-    // columns of B; barriers local to the CTA also in a pair).
+    // not FUSED: FP16 operand tiles, read by the MMA thread.  FUSED: FP32 tiles of A and B, which
+    // the converter warps turn into FP16 words in place (this CTA's own rows of A and its own
+    // columns of B; the "filled" barrier is local to the CTA also in a pair, the "free" barrier
+    // is the MMA thread's commit, which arrives in both CTAs).
     if (lane == 0) {
-      constexpr int RING = FUSED ? STAGES32 : STAGES;
+      constexpr int RING = STAGES;
       uint64_t* const ring_full = FUSED ? full32_bar : full_bar;
-      uint64_t* const ring_empty = FUSED ? empty32_bar : empty_bar;
+      uint64_t* const ring_empty = empty_bar;
       uint32_t it = 0;
       bool ok = true;
       auto load = [&](void* dst, const CUtensorMap* map, int x, int y, uint64_t* bar) {
@@ -815,20 +818,12 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA0, const __grid_constant__
           if constexpr (FUSED) {
             // A: one box {32 k (128 bytes), 128 rows}; B: boxes {32 columns (128 bytes), 32 k-rows}.
             // Rows and columns outside the matrices arrive as zeros, and split(0) = (0, 0).
-            uint8_t* st = smem32 + s * Cfg::STAGE32_BYTES;
-            mbar_arrive_expect_tx(&ring_full[s], Cfg::STAGE32_BYTES);
+            uint8_t* st = smem + s * Cfg::STAGE_BYTES;
+            mbar_arrive_expect_tx(&ring_full[s], Cfg::STAGE_BYTES);
             load(st, &tmA0, k0, tm * kBM, &ring_full[s]);
 #pragma unroll
             for (int a = 0; a < Cfg::BN_CTA / 32; ++a)
               load(st + Cfg::A32_TILE + a * (BK * 128), &tmB0, n0 + a * 32, k0, &ring_full[s]);
-#if SGC_L2_PREFETCH > 0
-            if (kb + SGC_L2_PREFETCH < kb1) {
-              const int kp = k0 + SGC_L2_PREFETCH * BK;
-              tma_prefetch_l2_2d(&tmA0, kp, tm * kBM);
-#pragma unroll
-              for (int a = 0; a < Cfg::BN_CTA / 32; ++a) tma_prefetch_l2_2d(&tmB0, n0 + a * 32, kp);
-            }
-#endif
           } else {
             uint8_t* st = smem + s * Cfg::STAGE_BYTES;
             // The leader announces the bytes of both CTAs' copies; the peer's copies may land first
@@ -883,37 +878,26 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA0, const __grid_constant__
   } else if (FUSED && warp >= kNumEpiWarps && warp < kNumEpiWarps + kNumConvWarps) {
     setmaxnreg_dec<88>();
     // ------------------------------------------------------------------ converter warps
-    // Per stage the FP32 ring holds A 128 x 32 (row m at m * 128 bytes, 16-byte chunk j of the row
-    // at position j ^ (m & 7): TMA's 128-byte swizzle) and B as BN_CTA / 32 boxes of 32 k-rows x
-    // 32 columns with the same row layout.  An item is 8 consecutive elements of a row (two
-    // chunks in, one hi chunk and one lo chunk out); a warp takes 32 items at a time:
-    //   A: 8 rows x 4 items.  Lane l: row l / 4, item l % 4.  A quarter warp reads 8 distinct
-    //      chunk positions (rows of both parities) and writes 128 contiguous bytes of the
-    //      64-byte-swizzled FP16 tile (row m at m * 64, chunk q at q ^ ((m >> 1) & 3)).
-    //   B: 2 k-rows (k even, k + 1) x 16 items, i.e. 128 columns.  Quarter warp w4, lanes 0-3:
-    //      row k, items 8 (w4 / 2) + 4 (w4 % 2) + 0..3; lanes 4-7: row k + 1, the other four items
-    //      of the same 64 columns.  Rows of both parities make the eight FP32 chunk positions
-    //      distinct, and the two groups of four land in complementary halves of a 128-byte row of
-    //      the FP16 atom (64 columns x 8 k-rows, chunk c at c ^ (k & 7)): no bank conflicts.
-    // Converter warp w takes A row blocks w, w + NW, ... and B row pairs w, w + NW, ... (both
-    // column halves when the CTA holds 256 columns), so (row & 7) and with it every swizzle term
-    // is a per-thread constant (NW a multiple of 4) and the rest of each address is an immediate.
+    // A stage is STAGE_BYTES / 1024 regions of 1 KB: 8 rows of 128 bytes (32 FP32 elements: 8 rows
+    // of A over 32 k, or 8 k-rows of B over 32 columns), 16-byte chunk j of row r at position
+    // j ^ r (TMA's 128-byte swizzle).  A warp converts a region in place: lane l takes the item
+    // (8 elements) q = l % 4 of row r = l / 4, reads its two chunks, and after the whole warp has
+    // read (__syncwarp) writes the hi chunk to r * 64 + ((q ^ (r / 2)) << 4) (rows of 64 bytes,
+    // 64-byte swizzle: the K-major atom of A, the MN-major atom of B) and the lo chunk 512 bytes
+    // further.  A quarter warp reads 8 distinct chunk positions (rows of both parities) and
+    // writes 128 contiguous bytes: no bank conflicts.  Warp w takes regions w, w + NW, ...; its
+    // offsets inside a region are per-thread constants and the rest of each address is an
+    // immediate.
     constexpr int NW = kNumConvWarps;
-    static_assert(NW % 4 == 0 && 16 % NW == 0, "converter warps: 4, 8 or 16");
-    constexpr int RA = 16 / NW;                       // A rounds per stage
-    constexpr int RB = 16 / NW;                       // B row-pair rounds per stage
-    constexpr int HC = Cfg::BN_CTA / 128;             // column halves
+    constexpr int kRegions = Cfg::STAGE_BYTES / 1024;             // 32 (pair) or 48
+    static_assert(kRegions % NW == 0, "regions per converter warp");
+    constexpr int R = kRegions / NW;
+    constexpr int kBatch = 4;                                     // regions loaded before converting
+    static_assert(R % kBatch == 0, "batches");
     const int cw = warp - kNumEpiWarps;
     const int ar = lane >> 2, aq = lane & 3;
-    const uint32_t a_src_c = (uint32_t)(cw * 1024 + ar * 128 + (((2 * aq) ^ ar) << 4));
-    const uint32_t a_dst_c = (uint32_t)(cw * 512 + ar * 64 + ((aq ^ ((ar >> 1) & 3)) << 4));
-    const int w4 = lane >> 3, up = (lane >> 2) & 1, jj = lane & 3;
-    const int cl = 8 * (w4 >> 1) + 4 * ((w4 & 1) ^ up) + jj;      // item within the 128 columns
-    const int rowlow = ((2 * cw) & 7) | up;                       // (k-row & 7)
-    const uint32_t b_src_c = Cfg::A32_TILE +
-        (uint32_t)((cl >> 2) * (BK * 128) + (2 * cw + up) * 128 + (((2 * (cl & 3)) ^ rowlow) << 4));
-    const uint32_t b_dst_c = 2 * Cfg::A_TILE +
-        (uint32_t)((cl >> 3) * (BK * 128) + (2 * cw + up) * 128 + (((cl & 7) ^ rowlow) << 4));
+    const uint32_t src_c = (uint32_t)(cw * 1024 + ar * 128 + (((2 * aq) ^ ar) << 4));
+    const uint32_t dst_c = (uint32_t)(cw * 1024 + ar * 64 + ((aq ^ ((ar >> 1) & 3)) << 4));
     const int total_stages = (first_tile < num_tiles)
         ? ((num_tiles - first_tile + tile_stride - 1) / tile_stride) * num_kb : 0;
     ConvScale cs;
@@ -921,31 +905,21 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA0, const __grid_constant__
     cs.fast = p.scale <= 32768.f;
     asm("mov.b64 %0, {%1, %1};" : "=l"(cs.scale2) : "f"(p.scale));
     cs.neg_scale_h = __half_as_ushort(__float2half_rn(cs.fast ? -p.scale : -1.f));
-    const uint32_t ring16 = smem_u32(smem), ring32 = smem_u32(smem32);
+    const uint32_t ring = smem_u32(smem);
     const bool timed = (blockIdx.x == 0 && threadIdx.x == kNumEpiWarps * 32);
     const bool timed1 = (blockIdx.x == 1 && threadIdx.x == (kNumEpiWarps + kNumConvWarps - 1) * 32);
     (void)timed; (void)timed1;
-    auto convert_stage = [&](uint32_t st32, uint32_t st16, auto fast_tag) {
+    auto convert_stage = [&](uint32_t st, auto fast_tag) {
       constexpr bool FAST = decltype(fast_tag)::value;
-      // batches of RA (= RB) items: all loads of a batch are issued before its arithmetic
-      const uint32_t a0 = st32 + a_src_c, a1 = a0 ^ 16u, ad = st16 + a_dst_c;
-      {
-        ConvItem x[RA];
+      const uint32_t s0 = st + src_c, s1 = s0 ^ 16u, d = st + dst_c;
 #pragma unroll
-        for (int r = 0; r < RA; ++r) load_item(x[r], a0 + r * NW * 1024, a1 + r * NW * 1024);
+      for (int b = 0; b < R; b += kBatch) {
+        ConvItem x[kBatch];
 #pragma unroll
-        for (int r = 0; r < RA; ++r) convert_store<FAST>(x[r], ad + r * NW * 512, Cfg::A_TILE, cs);
-      }
-      const uint32_t b0 = st32 + b_src_c, b1 = b0 ^ 16u, bd = st16 + b_dst_c;
+        for (int r = 0; r < kBatch; ++r) load_item(x[r], s0 + (b + r) * NW * 1024, s1 + (b + r) * NW * 1024);
+        __syncwarp();       // every lane has read its part of these regions: they may be overwritten
 #pragma unroll
-      for (int hc = 0; hc < HC; ++hc) {
-        ConvItem x[RB];
-#pragma unroll
-        for (int r = 0; r < RB; ++r)
-          load_item(x[r], b0 + hc * 4 * (BK * 128) + r * NW * 256, b1 + hc * 4 * (BK * 128) + r * NW * 256);
-#pragma unroll
-        for (int r = 0; r < RB; ++r)
-          convert_store<FAST>(x[r], bd + hc * 2 * (BK * 128) + r * NW * 256, Cfg::B_TILE, cs);
+        for (int r = 0; r < kBatch; ++r) convert_store<FAST>(x[r], d + (b + r) * NW * 1024, 512, cs);
       }
     };
     for (int it = 0; it < total_stages; ++it) {
@@ -956,25 +930,16 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA0, const __grid_constant__
         if (!mbar_wait_bounded(&full32_bar[s], ph, abort_flag, p.err, kErrConvFullWait, peer_abort)) break;
         SGC_TADD(11, timed);
       }
-      {
-        SGC_T0();
-        if (!mbar_wait_bounded(&empty_bar[s], ph ^ 1, abort_flag, p.err, kErrConvEmptyWait, peer_abort)) break;
-        SGC_TADD(0, timed);
-      }
       SGC_T0();
-      const uint32_t st32 = ring32 + s * Cfg::STAGE32_BYTES, st16 = ring16 + s * Cfg::STAGE_BYTES;
-      if (cs.fast) convert_stage(st32, st16, std::true_type{});
-      else convert_stage(st32, st16, std::false_type{});
+      const uint32_t st = ring + s * Cfg::STAGE_BYTES;
+      if (cs.fast) convert_stage(st, std::true_type{});
+      else convert_stage(st, std::false_type{});
       SGC_TADD(1, timed);
-      // Hand the stage to the relay thread (which makes it visible to the tensor core) and the
-      // FP32 stage back to the TMA producer.
+      // Hand the stage to the relay thread, which makes it visible to the tensor core.
       {
         SGC_T0();
         __syncwarp();
-        if (lane == 0) {
-          mbar_arrive(&conv_bar[s]);
-          mbar_arrive(&empty32_bar[s]);
-        }
+        if (lane == 0) mbar_arrive(&conv_bar[s]);
         SGC_TADD(2, timed);
         SGC_TADD(15, timed1);
       }

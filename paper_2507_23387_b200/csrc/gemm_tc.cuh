@@ -50,6 +50,20 @@ constexpr int kTcThreads = 384;     // not FUSED: + TMA warp + MMA warp (+ 2 idl
 #ifndef SGC_RELAY_ARRIVE
 #define SGC_RELAY_ARRIVE 1
 #endif
+// FUSED register split between the accumulate warps and the rest (512 threads x 128 registers),
+// columns per TMEM load in the accumulate warps, regions a converter warp loads before converting
+#ifndef SGC_FUSED_EPI_REGS
+#define SGC_FUSED_EPI_REGS 208
+#endif
+#ifndef SGC_FUSED_OTHER_REGS
+#define SGC_FUSED_OTHER_REGS 48
+#endif
+#ifndef SGC_FUSED_GW
+#define SGC_FUSED_GW 64
+#endif
+#ifndef SGC_CONV_BATCH
+#define SGC_CONV_BATCH 2
+#endif
 #ifndef SGC_CONV_WARPS
 #define SGC_CONV_WARPS 4
 #endif
@@ -390,7 +404,7 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA0, const __grid_constant__
   // (256 x 168 + 256 x 88 = 65536).  Each setmaxnreg sits at the top of its role's branch so
   // that the code below it is compiled against the new limit.
   if (warp < kNumEpiWarps) {
-    if (FUSED) setmaxnreg_inc<168>();
+    if (FUSED) setmaxnreg_inc<SGC_FUSED_EPI_REGS>();
     else setmaxnreg_inc<208>();       // 384 threads x 168: 256 x 208 + 128 x 56 fits the pool
     // ------------------------------------------------------------------ accumulate / epilogue
     const int quarter = warp & 3;                 // TMEM lanes 32*quarter .. +31 (warp id mod 4)
@@ -403,7 +417,7 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA0, const __grid_constant__
     float S[128];
     // TMEM is read 64 columns at a time (fewer, longer loads: the tensor pipe is held up for as
     // long as a drain lasts, and the load latency is most of that), 16 where registers are tight.
-    constexpr int GW = FUSED ? 16 : 64;
+    constexpr int GW = FUSED ? SGC_FUSED_GW : 64;
     auto wait_tfull = [&](int r) -> bool {
       return mbar_wait_bounded(&tfull_bar[r], drains[r] & 1, abort_flag, p.err, kErrEpiTmemFullWait, peer_abort);
     };
@@ -590,7 +604,7 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA0, const __grid_constant__
       SGC_TADD(8, blockIdx.x == 0 && threadIdx.x == 0);
     }
   } else if (warp == kMmaWarp) {
-    if (FUSED) setmaxnreg_dec<88>();
+    if (FUSED) setmaxnreg_dec<SGC_FUSED_OTHER_REGS>();
     else setmaxnreg_dec<56>();
     // ------------------------------------------------------------------ MMA issuer
     if (lane == 0 && leader) {
@@ -782,7 +796,7 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA0, const __grid_constant__
       mbar_wait_bounded(drain_bar, 0, nullptr, p.err, kErrDrainWait);
     }
   } else if (warp == kProducerWarp) {
-    if (FUSED) setmaxnreg_dec<88>();
+    if (FUSED) setmaxnreg_dec<SGC_FUSED_OTHER_REGS>();
     else setmaxnreg_dec<56>();
     // ------------------------------------------------------------------ TMA producer
     // not FUSED: FP16 operand tiles, read by the MMA thread.  FUSED: FP32 tiles of A and B, which
@@ -876,7 +890,7 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA0, const __grid_constant__
       }
     }
   } else if (FUSED && warp >= kNumEpiWarps && warp < kNumEpiWarps + kNumConvWarps) {
-    setmaxnreg_dec<88>();
+    setmaxnreg_dec<SGC_FUSED_OTHER_REGS>();
     // ------------------------------------------------------------------ converter warps
     // A stage is STAGE_BYTES / 1024 regions of 1 KB: 8 rows of 128 bytes (32 FP32 elements: 8 rows
     // of A over 32 k, or 8 k-rows of B over 32 columns), 16-byte chunk j of row r at position
@@ -892,7 +906,7 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA0, const __grid_constant__
     constexpr int kRegions = Cfg::STAGE_BYTES / 1024;             // 32 (pair) or 48
     static_assert(kRegions % NW == 0, "regions per converter warp");
     constexpr int R = kRegions / NW;
-    constexpr int kBatch = 4;                                     // regions loaded before converting
+    constexpr int kBatch = SGC_CONV_BATCH;                                     // regions loaded before converting
     static_assert(R % kBatch == 0, "batches");
     const int cw = warp - kNumEpiWarps;
     const int ar = lane >> 2, aq = lane & 3;
@@ -948,7 +962,7 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA0, const __grid_constant__
 #endif
     }
   } else if (FUSED) {
-    setmaxnreg_dec<88>();
+    setmaxnreg_dec<SGC_FUSED_OTHER_REGS>();
     // ------------------------------------------------------------------ relay threads
     // The converters' stores go through the generic proxy and the tensor core reads through the
     // async proxy, so a proxy fence has to lie between the two.  Inside a cluster that fence

@@ -79,15 +79,16 @@ enum {
    * tcgen05.mma.cta_group::2 (256 x 256 tile per pair, each CTA loading half of the B tile);
    * 0: one CTA per 128 x 256 tile; 2 (default): the library chooses: pairs for the kernels that
    * read FP16 words (two-phase sgemm_cube, sgemm_cube_presplit, sgemm_cube_hgemm, ...) whenever
-   * M > 128 and split-K (below, single CTAs only) does not apply, single CTAs for the fused
-   * converter kernel.  Same arithmetic, bit-identical results either way as long as split-K does
-   * not apply.  (Pairs pull two thirds of the bytes of single CTAs from L2 into the SMs, which is
+   * M > 128 and split-K (below, single CTAs only) does not apply, and for the fused converter
+   * kernel whenever M > 128.  Same arithmetic, bit-identical results either way as long as
+   * split-K does not apply.  (Pairs pull two thirds of the bytes of single CTAs from L2 into the SMs, which is
    * what bounds this kernel: 458 against 439 TFLOP/s at 8192^3, 407 against 378 at 4096^3.) */
   SGEMM_CUBE_OPT_CTA_PAIR = 2,
   /* How sgemm_cube computes (same arithmetic; same bracketing and bit-identical results except
    * where split-K, which only the two-phase strategy uses, re-brackets the k-block sums):
-   * SGEMM_CUBE_STRATEGY_FUSED     one kernel; converter warps split FP32 tiles on the fly, no FP16
-   *                               copy of A or B exists in device memory, no workspace;
+   * SGEMM_CUBE_STRATEGY_FUSED     one kernel; TMA stages FP32 tiles in shared memory, converter
+   *                               warps split them there in place, no FP16 copy of A or B exists
+   *                               in device memory, no workspace;
    * SGEMM_CUBE_STRATEGY_TWO_PHASE the split kernel writes the FP16 words of A and B once into the
    *                               handle's workspace (4 bytes per element of A and B, grown with
    *                               cudaMalloc on first use), then one kernel forms all three
@@ -207,8 +208,9 @@ int sgemm_cube_hgemm(sgemm_cube_handle h, int M, int N, int K,
                      float* D_dev, int64_t ldd, int accumulate, void* stream);
 
 /* Host-buffer convenience around sgemm_cube: copies A and B from HOST memory to the handle's
- * device workspace, runs the fused kernel, copies C back to HOST memory and synchronises the
- * stream before returning.  Pinned host memory makes the copies asynchronous to the host but the
+ * device workspace, runs the computation of sgemm_cube there (same strategy choice, see
+ * SGEMM_CUBE_OPT_STRATEGY), copies C back to HOST memory and synchronises the stream before
+ * returning.  Pinned host memory makes the copies asynchronous to the host but the
  * call still returns only when C_host is complete.  For M >= 1024 and M*N*K >= 2^30 (and a
  * strategy other than FUSED) the call is pipelined: B is copied and split once, A and C move in
  * about eight row panels on two internal copy streams so that the upload of one panel, the
@@ -353,11 +355,17 @@ int sgemm_cube_auto_scaled(sgemm_cube_handle h, int M, int N, int K,
  *   Arguments, layouts and alignment as sgemm_cube_unfused, on the CURRENT device
  *   (A_dev, B_dev, C_dev must be on it).
  *   The first call on a device looks up the array's device address and configures the kernels;
- *   make that first call outside any stream capture.  Later calls only launch.
+ *   make that first call outside any stream capture, and at start-up: the 32 MiB are committed
+ *   when the CUDA runtime loads the library's device code on that GPU, which with lazy module
+ *   loading can be as late as this first call, so a process whose device memory is already
+ *   exhausted gets CUDA_ERROR from it.  Later calls only launch and leave the amount of free
+ *   device memory unchanged.
  *   All calls share the one array, which keeps whatever the last call left in it.  Every region a
  *   call reads is first overwritten by that call, so results never depend on earlier calls; but
  *   two calls that may overlap on the GPU (different streams without an ordering between them,
- *   or different host threads) race on the scratch and give undefined results.
+ *   whether from one host thread or several) race on the scratch and give undefined results.
+ *   Host threads may call concurrently as far as the host side goes (enqueueing is serialised
+ *   internally).
  *   A kernel-side bounded-wait failure (never expected) cannot be reported by this entry point;
  *   C is then unspecified.
  * Errors: INVALID_ARG, TOO_LARGE, UNSUPPORTED_ARCH, CUDA_ERROR. */
@@ -386,6 +394,30 @@ int sgemm_cube_last_kernel_ms(sgemm_cube_handle h, float* ms_out);
  * how many calls were averaged.  Waits for those kernels to finish, then starts a new average.
  * Errors: INVALID_ARG (timing off, or no call since), CUDA_ERROR. */
 int sgemm_cube_mean_kernel_ms(sgemm_cube_handle h, float* mean_ms_out, int* calls_out);
+
+/* SM clock cycles and nanoseconds (device global timer) that the tensor-core kernel of the most
+ * recent sgemm_cube call ran for, taken inside the kernel by its first CTA (requires
+ * SGEMM_CUBE_OPT_TIME_KERNEL = 1 before that call; waits for the device to finish).  Their
+ * quotient is the SM clock the kernel actually ran at, which under a power cap is well below the
+ * clock that nvidia-smi shows between kernels; the three-GEMM roofline at that clock is
+ * SMs x 8192 FP16 flop/clk x (cycles / ns) / 3.
+ * Errors: INVALID_ARG (timing off), CUDA_ERROR. */
+int sgemm_cube_last_kernel_clock(sgemm_cube_handle h, uint64_t* sm_cycles_out, uint64_t* ns_out);
+
+/* ---- Diagnostics for the failure-reporting path (tests; nothing on the GEMM path calls them).
+ * Every wait inside the kernels is bounded; a wait that runs out writes a code into the handle's
+ * device error word, the CTA drains and exits, and sgemm_cube_check / sgemm_cube_destroy report
+ * SGEMM_CUBE_DEVICE_TIMEOUT.  Neither function below makes a GEMM kernel fail.
+ *
+ * sgemm_cube_debug_inject_error: host-made failure.  Waits for the device, then copies `code`
+ * into the error word, as if a kernel had recorded it.
+ * sgemm_cube_debug_wait_timeout: enqueues a one-CTA kernel in which one thread runs the kernels'
+ * bounded wait, with a limit of `limit_clocks` SM clocks (1 .. 10^8), on a barrier that nothing
+ * signals; the wait gives up after the limit and records code 0x1F0.  The kernel then ends
+ * normally and the context stays usable.
+ * Errors: INVALID_ARG, CUDA_ERROR. */
+int sgemm_cube_debug_inject_error(sgemm_cube_handle h, uint32_t code);
+int sgemm_cube_debug_wait_timeout(sgemm_cube_handle h, int64_t limit_clocks, void* stream);
 
 /* Text for a status code (static storage; never NULL). */
 const char* sgemm_cube_status_string(int status);

@@ -24,6 +24,7 @@ EXPORTS = ["sgemm_cube_create", "sgemm_cube_destroy", "sgemm_cube_set_option", "
            "sgemm_cube_scaled", "sgemm_cube_auto_scaled",
            "sgemm_cube_host", "sgemm_cube_unfused_static", "sgemm_cube_check", "sgemm_cube_launch_count", "sgemm_cube_last_kernel_ms", "sgemm_cube_mean_kernel_ms",
            "sgemm_cube_exponent_window", "sgemm_cube_choose_scale_exp", "sgemm_cube_residual_overflow_count",
+           "sgemm_cube_last_kernel_clock", "sgemm_cube_debug_inject_error", "sgemm_cube_debug_wait_timeout",
            "sgemm_cube_status_string", "sgemm_cube_version"]
 
 _lib = None
@@ -70,6 +71,10 @@ def load():
     lib.sgemm_cube_residual_overflow_count.argtypes = [vp, i32, i32, vp, vp, i64, ctypes.POINTER(i64), vp]
     lib.sgemm_cube_choose_scale_exp.argtypes = [ctypes.POINTER(i64), ctypes.POINTER(i64),
                                                 ctypes.POINTER(i32), ctypes.POINTER(i32)]
+    lib.sgemm_cube_last_kernel_clock.argtypes = [vp, ctypes.POINTER(ctypes.c_uint64),
+                                                 ctypes.POINTER(ctypes.c_uint64)]
+    lib.sgemm_cube_debug_inject_error.argtypes = [vp, ctypes.c_uint32]
+    lib.sgemm_cube_debug_wait_timeout.argtypes = [vp, i64, vp]
     lib.sgemm_cube_launch_count.argtypes = [vp]
     lib.sgemm_cube_launch_count.restype = i64
     lib.sgemm_cube_status_string.argtypes = [i32]
@@ -298,3 +303,18 @@ class Handle:
         _check(load().sgemm_cube_mean_kernel_ms(self._h, ctypes.byref(ms), ctypes.byref(n)),
                "sgemm_cube_mean_kernel_ms")
         return float(ms.value), int(n.value)
+
+    def sgemm_cube_last_kernel_clock(self):
+        """(SM cycles, nanoseconds) the tensor-core kernel of the last timed sgemm_cube call ran for."""
+        cyc, ns = ctypes.c_uint64(0), ctypes.c_uint64(0)
+        _check(load().sgemm_cube_last_kernel_clock(self._h, ctypes.byref(cyc), ctypes.byref(ns)),
+               "sgemm_cube_last_kernel_clock")
+        return int(cyc.value), int(ns.value)
+
+    def sgemm_cube_debug_inject_error(self, code: int):
+        _check(load().sgemm_cube_debug_inject_error(self._h, ctypes.c_uint32(code)),
+               "sgemm_cube_debug_inject_error")
+
+    def sgemm_cube_debug_wait_timeout(self, limit_clocks: int, stream=None):
+        _check(load().sgemm_cube_debug_wait_timeout(self._h, ctypes.c_int64(limit_clocks),
+                                                    _stream_ptr(stream)), "sgemm_cube_debug_wait_timeout")

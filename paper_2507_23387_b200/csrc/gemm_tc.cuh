@@ -82,6 +82,7 @@ enum : unsigned int {
   kErrConvEmptyWait = 0x106,
   kErrConvFullWait = 0x107,
   kErrRelayWait = 0x108,
+  kErrProbeWait = 0x1F0,
 };
 
 // Optional role timing (compile with -DSGC_ROLE_TIMING): CTA 0 adds the clocks each role spends in
@@ -122,6 +123,9 @@ struct TcGemmParams {
   float* Px;
   long long pstride;
   long long ldp;
+  // Optional (may be null): thread 0 of CTA 0 stores how long it ran, {SM clocks, nanoseconds of
+  // the global timer}, from which the host gets the SM clock the kernel actually ran at.
+  unsigned long long* kclock;
 };
 
 #ifndef SGC_PAIR_GROUP
@@ -337,6 +341,13 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA0, const __grid_constant__
 
   const int warp = threadIdx.x >> 5;
   const int lane = threadIdx.x & 31;
+  long long kclock_clk0 = 0;
+  unsigned long long kclock_ns0 = 0;
+  const bool kclock_on = (p.kclock != nullptr) && blockIdx.x == 0 && threadIdx.x == 0;
+  if (kclock_on) {
+    kclock_clk0 = clock64();
+    asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(kclock_ns0));
+  }
 #ifdef SGC_ROLE_TIMING
   long long sgc_k_clk0 = 0;
   unsigned long long sgc_k_ns0 = 0;
@@ -1001,6 +1012,12 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA0, const __grid_constant__
   // ---------------------------------------------------------------------- teardown
   tc_fence_before_sync();
   __syncthreads();
+  if (kclock_on) {
+    unsigned long long ns1;
+    asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(ns1));
+    p.kclock[0] = (unsigned long long)(clock64() - kclock_clk0);
+    p.kclock[1] = ns1 - kclock_ns0;
+  }
 #ifdef SGC_ROLE_TIMING
   if (blockIdx.x == 0 && threadIdx.x == 0) {
     unsigned long long ns1;
@@ -1016,6 +1033,25 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA0, const __grid_constant__
     if (PAIR) tmem_dealloc_pair(tmem_base, kTmemCols);
     else tmem_dealloc(tmem_base, kTmemCols);
   }
+}
+
+// Diagnostic kernel (one CTA): thread 0 waits, with the bounded wait that every role of the
+// kernels above uses, on an mbarrier that nothing ever signals, so the wait runs into its clock
+// limit, publishes kErrProbeWait in the error word and raises the CTA's abort flag; the second
+// warp waits on the same barrier with the full limit and must leave as soon as the flag is up.
+// Lets a test walk the path device wait -> error word -> host status without making any real
+// pipeline fail.  `limit` is a few thousand clocks.
+__global__ void wait_timeout_probe_kernel(unsigned int* err, long long limit) {
+  __shared__ uint64_t bar;
+  __shared__ uint32_t abort_flag;
+  if (threadIdx.x == 0) {
+    mbar_init(&bar, 1);
+    abort_flag = 0u;
+    fence_mbar_init();
+  }
+  __syncthreads();
+  if (threadIdx.x == 0) mbar_wait_bounded(&bar, 0, &abort_flag, err, kErrProbeWait, 0u, limit);
+  if (threadIdx.x == 32) mbar_wait_bounded(&bar, 0, &abort_flag, err, kErrProbeWait + 1, 0u, kWaitLimitClocks);
 }
 
 }  // namespace sgc

@@ -41,7 +41,9 @@ inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 
 struct sgemm_cube_ctx {
   int device = 0;
   int sm_count = 0;
-  unsigned int* err_dev = nullptr;   // [0] error word; [4..8] scratch of sgemm_cube_exponent_window
+  unsigned int* err_dev = nullptr;   // [0] error word; [4..13] scratch of sgemm_cube_exponent_window;
+                                     // [16..19] clocks and nanoseconds of the last timed tensor-core kernel
+  bool err_dev_has_clock = false;    // false for the static entry point's single error word
   void* ws = nullptr;          // unfused path: FP16 words of A and B, D_hh, D_x
   size_t ws_bytes = 0;
   void* part_ws = nullptr;     // split-K partial sums
@@ -301,6 +303,8 @@ int launch_tc_gemm(sgemm_cube_ctx* h, int M, int N, int K, const uint16_t* Ahi, 
   p.err = h->err_dev;
   p.A32 = nullptr; p.lda32 = 0; p.B32 = nullptr; p.ldb32 = 0; p.scale = 1.f;
   p.ksplit = 1; p.kslice_blocks = 0; p.Phh = nullptr; p.Px = nullptr; p.pstride = 0; p.ldp = 0;
+  p.kclock = (NTERMS == 3 && h->time_kernel && h->err_dev_has_clock)
+                 ? reinterpret_cast<unsigned long long*>(h->err_dev + 16) : nullptr;
   // Split-K: when the tiles would leave more than half of the SMs idle and k is long, cut the k
   // range into slices (whole k-blocks) so that tiles x slices fills the machine; a reduction
   // kernel adds the slices' sums.
@@ -383,6 +387,8 @@ int launch_fused(sgemm_cube_ctx* h, int M, int N, int K, const float* A, int64_t
   p.B32 = B; p.ldb32 = ldb;
   p.scale = ldexpf(1.0f, s);
   p.ksplit = 1; p.kslice_blocks = 0; p.Phh = nullptr; p.Px = nullptr; p.pstride = 0; p.ldp = 0;
+  p.kclock = (h->time_kernel && h->err_dev_has_clock)
+                 ? reinterpret_cast<unsigned long long*>(h->err_dev + 16) : nullptr;
   // FP32 tiles as TMA stages them for the converter warps: A in boxes of {BK k, 128 rows}, B in
   // boxes of {32 columns, BK k-rows}, both with the 128-byte swizzle (rows of 128 bytes).
   CUtensorMap tmA, tmB;
@@ -495,16 +501,17 @@ int sgemm_cube_create(sgemm_cube_handle* out, int device) {
     return SGEMM_CUBE_CUDA_ERROR;
   }
   h->encode = reinterpret_cast<EncodeTiledFn>(fn);
-  if (cudaMalloc(reinterpret_cast<void**>(&h->err_dev), 16 * sizeof(unsigned int)) != cudaSuccess) {
+  if (cudaMalloc(reinterpret_cast<void**>(&h->err_dev), 32 * sizeof(unsigned int)) != cudaSuccess) {
     cudaGetLastError();
     delete h;
     return SGEMM_CUBE_ALLOC_FAILED;
   }
-  if (cudaMemset(h->err_dev, 0, 16 * sizeof(unsigned int)) != cudaSuccess) {
+  if (cudaMemset(h->err_dev, 0, 32 * sizeof(unsigned int)) != cudaSuccess) {
     cudaFree(h->err_dev);
     delete h;
     return SGEMM_CUBE_CUDA_ERROR;
   }
+  h->err_dev_has_clock = true;
   *out = h;
   return SGEMM_CUBE_OK;
 }
@@ -1089,6 +1096,43 @@ int sgemm_cube_mean_kernel_ms(sgemm_cube_handle h, float* mean_ms_out, int* call
   return SGEMM_CUBE_OK;
 }
 
+int sgemm_cube_last_kernel_clock(sgemm_cube_handle h, uint64_t* sm_cycles_out, uint64_t* ns_out) {
+  if (!h || !sm_cycles_out || !ns_out || !h->time_kernel || !h->err_dev_has_clock) return SGEMM_CUBE_INVALID_ARG;
+  DeviceGuard g(h->device);
+  if (!g.ok) return SGEMM_CUBE_CUDA_ERROR;
+  unsigned long long v[2] = {0, 0};
+  if (cudaDeviceSynchronize() != cudaSuccess ||
+      cudaMemcpy(v, h->err_dev + 16, sizeof(v), cudaMemcpyDeviceToHost) != cudaSuccess) {
+    cudaGetLastError();
+    return SGEMM_CUBE_CUDA_ERROR;
+  }
+  *sm_cycles_out = v[0];
+  *ns_out = v[1];
+  return SGEMM_CUBE_OK;
+}
+
+int sgemm_cube_debug_inject_error(sgemm_cube_handle h, uint32_t code) {
+  if (!h) return SGEMM_CUBE_INVALID_ARG;
+  DeviceGuard g(h->device);
+  if (!g.ok) return SGEMM_CUBE_CUDA_ERROR;
+  if (cudaDeviceSynchronize() != cudaSuccess ||
+      cudaMemcpy(h->err_dev, &code, sizeof(code), cudaMemcpyHostToDevice) != cudaSuccess) {
+    cudaGetLastError();
+    return SGEMM_CUBE_CUDA_ERROR;
+  }
+  return SGEMM_CUBE_OK;
+}
+
+int sgemm_cube_debug_wait_timeout(sgemm_cube_handle h, int64_t limit_clocks, void* stream) {
+  if (!h || limit_clocks < 1 || limit_clocks > 100000000) return SGEMM_CUBE_INVALID_ARG;
+  DeviceGuard g(h->device);
+  if (!g.ok) return SGEMM_CUBE_CUDA_ERROR;
+  sgc::wait_timeout_probe_kernel<<<1, 32, 0, static_cast<cudaStream_t>(stream)>>>(h->err_dev,
+                                                                                (long long)limit_clocks);
+  h->launches++;
+  return cudaGetLastError() == cudaSuccess ? SGEMM_CUBE_OK : SGEMM_CUBE_CUDA_ERROR;
+}
+
 }  // extern "C"
 
 // ---------------------------------------------------------------------------------------------
@@ -1177,6 +1221,9 @@ extern "C" int sgemm_cube_unfused_static(int M, int N, int K, const float* A, in
   rc = static_setup(device, &s);
   if (rc) return rc;
   sgemm_cube_ctx* h = &s->ctx;
+  // The per-device launch state is shared by every caller of this entry point: host threads
+  // enqueue one at a time (the GPU work itself is ordered by the caller's streams).
+  std::lock_guard<std::mutex> lock(g_static_mutex);
   cudaStream_t st = static_cast<cudaStream_t>(stream);
   unsigned char* w = s->scratch;
   uint16_t* Ahi = reinterpret_cast<uint16_t*>(w);

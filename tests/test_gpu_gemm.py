@@ -164,6 +164,77 @@ def test_strategies_agree_bitwise(handle):
         assert np.array_equal(C1, C2) and np.array_equal(C1, C3)
 
 
+@pytest.mark.parametrize("n", [4096, 8192])
+def test_strategies_and_cta_modes_agree_on_the_full_matrix(handle, n):
+    """Several waves of the persistent grid, the partly filled last wave included: the fused
+    kernel, the two-phase route and the pre-split entry point, each with CTA pairs and with single
+    CTAs, must produce the same M x N matrix bit for bit (compared on the device, every element).
+    What that common result is worth is checked against the oracle on the rows of tile_rows()."""
+    A, B = inputs.make_pair("exponent_spread", 0, n, n, n)
+    Ad, Bd = to_dev(A), to_dev(B)
+    rows = tile_rows(n)
+    ref = {}
+    try:
+        handle.sgemm_cube_set_option(binding.OPT_SPLIT_K, 0)
+        for order in (T, E):
+            for strategy in ("two_phase", "fused"):
+                for pair in (1, 0):
+                    handle.sgemm_cube_set_option(binding.OPT_CTA_PAIR, pair)
+                    handle.sgemm_cube_set_option(binding.OPT_STRATEGY, STRATEGY[strategy])
+                    C = torch.full((n, n), float("nan"), device="cuda:0")
+                    handle.sgemm_cube(Ad, Bd, C, 11, order)
+                    st, det = handle.sgemm_cube_check()
+                    assert st == 0, hex(det)
+                    if order not in ref:
+                        ref[order] = C
+                        gates(C[torch.as_tensor(rows, device="cuda:0")].cpu().numpy(), A[rows], B, 11, order,
+                              label="%d^3 order %d" % (n, order))
+                    else:
+                        assert torch.equal(C, ref[order]), (n, order, strategy, pair)
+                    del C
+    finally:
+        handle.sgemm_cube_set_option(binding.OPT_CTA_PAIR, 2)
+        handle.sgemm_cube_set_option(binding.OPT_SPLIT_K, 1)
+        handle.sgemm_cube_set_option(binding.OPT_STRATEGY, binding.STRATEGY_AUTO)
+
+
+@pytest.mark.parametrize("path,order", PATHS + [("fused", binding.ELEMENTWISE_REORDERED),
+                                                ("two_phase", binding.ELEMENTWISE_REORDERED)])
+@pytest.mark.parametrize("kblock", [64, 128])
+def test_residual_carrying_inputs_exact_over_several_stages_and_k_blocks(handle, path, order, kblock):
+    """Entries +-(1 + q 2^-13), q in {-1, 0, 1}: hi = +-1 and lo = +-q 2^-2 (s = 11), so every
+    product and every partial sum of every stream is a small multiple of a power of two and no
+    addition rounds, on the tensor core or off it.  With K = 448 (seven 64-deep stages, 3.5
+    k-blocks of 128) the look-ahead at the start of a k-block, the swapped last stage, the k-block
+    drains and the ragged last k-block all carry non-zero lo words, and every path must reproduce
+    the oracle (Eq. recover_eqn with Eq. termwise / Eq. elementwise) bit for bit."""
+    rng = np.random.default_rng(7)
+    M, N, K = 384, 520, 448
+    def draw(shape):
+        q = rng.integers(-1, 2, size=shape).astype(np.float64)
+        sgn = rng.choice([-1.0, 1.0], size=shape)
+        return (sgn * (1.0 + q * 2.0 ** -13)).astype(np.float32)
+    A, B = draw((M, K)), draw((K, N))
+    opt = binding.OPT_TERMWISE_K_BLOCK if order == T else binding.OPT_ELEMENTWISE_K_BLOCK
+    want = oracle.sgemm_cube(A, B, 11, order, kblock)
+    # exact value of the three kept terms, from the words themselves
+    hiA, loA = oracle.split(A, 11)
+    hiB, loB = oracle.split(B, 11)
+    f = lambda w: oracle.f16_to_f32(w).view(np.float32).astype(np.float64)
+    exact = f(hiA) @ f(hiB) + (f(loA) @ f(hiB) + f(hiA) @ f(loB)) * 2.0 ** -11
+    assert np.array_equal(want.astype(np.float64), exact)
+    assert np.any(f(loA) != 0) and np.any(f(loB) != 0)
+    try:
+        handle.sgemm_cube_set_option(opt, kblock)
+        for pair in (1, 0):
+            handle.sgemm_cube_set_option(binding.OPT_CTA_PAIR, pair)
+            C = run(handle, path, padded_dev(A, 4), padded_dev(B, 4), 11, order)
+            assert np.array_equal(C, want), (path, order, kblock, pair)
+    finally:
+        handle.sgemm_cube_set_option(binding.OPT_CTA_PAIR, 2)
+        handle.sgemm_cube_set_option(opt, K_BLOCK[order])
+
+
 @pytest.mark.parametrize("path,order", PATHS)
 def test_cta_pair_mode_is_bit_identical(handle, path, order):
     # tcgen05.mma.cta_group::2 (two CTAs per 256 x 256 tile) against one CTA per 128 x 256 tile.
@@ -222,6 +293,17 @@ def test_k_block_option_changes_bracketing_not_validity(handle):
         handle.sgemm_cube_set_option(binding.OPT_TERMWISE_K_BLOCK, 100)
 
 
+def tile_rows(M, extra=0, seed=0):
+    """One row out of every 128-row block of the result (so every row tile, both CTAs of every
+    256-row pair tile and, since whole rows are compared, every column tile and every wave of the
+    persistent grid is looked at), at an offset inside the block that changes from block to block
+    (all four lane quarters of the accumulator), plus `extra` random rows."""
+    rows = {min(M - 1, b * 128 + (b * 37 + 5) % 128) for b in range((M + 127) // 128)}
+    if extra:
+        rows |= set(np.random.default_rng(seed).choice(M, extra, replace=False).tolist())
+    return np.array(sorted(rows))
+
+
 def _sampled_rows_check(handle, path, order, A_rows_np, B_np, C_dev, rows, label):
     C_rows = C_dev[torch.as_tensor(rows, device="cuda:0")].cpu().numpy()
     return gates(C_rows, A_rows_np, B_np, 11, order, label=label)
@@ -231,9 +313,8 @@ def _sampled_rows_check(handle, path, order, A_rows_np, B_np, C_dev, rows, label
 def test_config2_4096_cubed_sampled_rows(handle, path, order):
     n = 4096
     A, B = inputs.make_pair("uniform_pm1", 0, n, n, n)
-    rows = np.sort(np.random.default_rng(0).choice(n, 48, replace=False))
+    rows = tile_rows(n, extra=16, seed=0)
     Ad, Bd = to_dev(A), to_dev(B)
-    C = torch.empty((n, n), device="cuda:0")
     C = torch.from_numpy(run(handle, path, Ad, Bd, 11, order)).to("cuda:0")
     _sampled_rows_check(handle, path, order, A[rows], B, C, rows, "4096^3 %s %d" % (path, order))
 
@@ -260,7 +341,7 @@ def test_config2_orders_compared(handle):
 def test_config3_8192_cubed_exponent_spread_sampled_rows(handle, path, order):
     n = 8192
     A, B = inputs.make_pair("exponent_spread", 0, n, n, n)
-    rows = np.sort(np.random.default_rng(1).choice(n, 24, replace=False))
+    rows = tile_rows(n)
     Ad, Bd = to_dev(A), to_dev(B)
     C = torch.from_numpy(run(handle, path, Ad, Bd, 11, order))
     gates(C[torch.as_tensor(rows)].numpy(), A[rows], B, 11, order, label="8192^3 %s" % path)
@@ -302,7 +383,7 @@ def test_config5_large_shapes_sampled_rows(handle, shape):
     C = torch.empty((M, N), device="cuda:0")
     handle.sgemm_cube(A, B, C, 11, T)
     assert handle.sgemm_cube_check()[0] == 0
-    rows = np.sort(np.random.default_rng(2).choice(M, 8, replace=False))
+    rows = tile_rows(M)
     idx = torch.as_tensor(rows, device="cuda:0")
     gates(C[idx].cpu().numpy(), A[idx].cpu().numpy(), B.cpu().numpy(), 11, T, label=str(shape))
     # properties that hold at any size: a permutation of A's rows permutes C's rows exactly

@@ -302,3 +302,62 @@ def test_leading_dimensions_are_honoured():
     C1 = oracle.sgemm_cube(A, B, kb=8)
     C2 = oracle.sgemm_cube(np.ascontiguousarray(A), np.ascontiguousarray(B), kb=8)
     assert np.array_equal(C1, C2)
+
+
+# ------------------------------------------------------------------ metric helpers, by hand
+def test_error_metrics_on_cases_worked_by_hand():
+    """componentwise_err = max |C - C64| / (|A||B|) (the measure Eq. main_bound is stated in) and
+    frobenius_rel_err = ||C - C64||_F / ||C64||_F (Eq. err), on 2 x 2 cases small enough to do on
+    paper.  A = [[1, -2], [0, 4]], B = [[3, 1], [1, -1]]:
+        C64    = [[1, 3], [4, -4]]         |A||B| = [[5, 3], [4, 4]]   (differs from |C64|)
+    and a result that is off by [[0.5, 0], [0, -1]]."""
+    C64 = np.array([[1.0, 3.0], [4.0, -4.0]])
+    AB = np.array([[5.0, 3.0], [4.0, 4.0]])
+    A = np.array([[1, -2], [0, 4]], dtype=np.float32)
+    B = np.array([[3, 1], [1, -1]], dtype=np.float32)
+    C64_o, AB_o = oracle.dgemm_ref(A, B)
+    assert np.array_equal(C64_o, C64) and np.array_equal(AB_o, AB)
+    C = C64 + np.array([[0.5, 0.0], [0.0, -1.0]])
+    # componentwise: max(0.5 / 5, 1 / 4) = 0.25; dividing by |C64| instead would give 0.5
+    assert oracle.componentwise_err(C, C64, AB) == 0.25
+    # Frobenius: sqrt(0.25 + 1) / sqrt(1 + 9 + 16 + 16) = sqrt(1.25 / 42); without the square
+    # roots it would be 1.25 / 42
+    assert oracle.frobenius_rel_err(C, C64) == pytest.approx((1.25 / 42.0) ** 0.5, rel=1e-15)
+    assert oracle.frobenius_rel_err(C64, C64) == 0.0 and oracle.componentwise_err(C64, C64, AB) == 0.0
+    # the largest quotient decides, not the largest difference
+    C2 = C64 + np.array([[1.0, 0.9], [0.0, 0.0]])            # quotients 0.2 and 0.3
+    assert oracle.componentwise_err(C2, C64, AB) == pytest.approx(0.3, rel=1e-15)
+
+
+def test_componentwise_error_where_the_bound_is_zero():
+    """An entry with (|A||B|)_ij = 0 has no tolerance at all: every product in it is zero, so any
+    non-zero result there is an infinite error, and a zero result does not count."""
+    A = np.array([[0, 0], [1, 2]], dtype=np.float32)
+    B = np.array([[1, 0], [1, 0]], dtype=np.float32)          # |A||B| = [[0, 0], [3, 0]]
+    C64, AB = oracle.dgemm_ref(A, B)
+    assert np.array_equal(AB, np.array([[0.0, 0.0], [3.0, 0.0]]))
+    good = np.array([[0.0, 0.0], [3.75, 0.0]])
+    assert oracle.componentwise_err(good, C64, AB) == 0.25
+    bad = good.copy()
+    bad[0, 1] = 1e-30
+    assert oracle.componentwise_err(bad, C64, AB) == float("inf")
+    assert oracle.componentwise_err(np.zeros((1, 2)), np.zeros((1, 2)), np.zeros((1, 2))) == 0.0
+
+
+def test_sgemm_f32_rounds_every_addition_to_fp32_in_k_order():
+    """oracle.sgemm_f32 is the plain FP32 GEMM: products rounded to FP32, then added one after the
+    other in ascending k with a rounding after each addition.  Brute force with exact rationals
+    and the explicit rounding step above; K = 7 on inputs whose partial sums are not exact, so an
+    implementation that accumulates in double (or in another order) gives different bits."""
+    A, B = inputs.make_pair("normal", 3, 4, 5, 7)
+    C = oracle.sgemm_f32(A, B)
+    for i in range(A.shape[0]):
+        for j in range(B.shape[1]):
+            acc = Fraction(0)
+            for k in range(A.shape[1]):
+                prod = _rn32(Fraction(float(A[i, k])) * Fraction(float(B[k, j])))
+                acc = _rn32(acc + prod)
+            assert Fraction(float(C[i, j])) == acc, (i, j)
+    # the two accumulation precisions really differ on this input
+    C_double = (A.astype(np.float64) @ B.astype(np.float64)).astype(np.float32)
+    assert not np.array_equal(C, C_double)

@@ -40,6 +40,24 @@ def test_static_scratch_variant_matches_allocating_variant_twice_in_a_row():
         h.destroy()
 
 
+def test_static_scratch_variant_leaves_free_device_memory_unchanged():
+    """What the entry point is for: after its first (set-up) call on a device, a call takes no
+    device memory.  Measured with the driver's own free-memory figure around a call, with the
+    inputs and the output allocated beforehand (so that torch's allocator is not involved)."""
+    torch.cuda.set_device(0)
+    A, B = _pair(5, 512, 384, 256)
+    C = torch.empty((512, 384), device="cuda:0")
+    binding.sgemm_cube_unfused_static(A, B, C, 11)        # set-up call (the first one on this device, if no test ran before)
+    torch.cuda.synchronize()
+    free_before, _ = torch.cuda.mem_get_info(0)
+    for _ in range(3):
+        binding.sgemm_cube_unfused_static(A, B, C, 11)
+    torch.cuda.synchronize()
+    free_after, _ = torch.cuda.mem_get_info(0)
+    assert free_after == free_before
+    assert torch.isfinite(C).all()
+
+
 def test_static_scratch_variant_rejects_what_does_not_fit():
     torch.cuda.set_device(0)
     M = N = K = 2048                      # needs 64 MiB of scratch; the array has 32 MiB

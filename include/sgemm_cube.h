@@ -10,9 +10,9 @@
  *
  *      C  ~=  hi_A hi_B  +  2^-s ( lo_A hi_B  +  hi_A lo_B )
  *
- * (paper: Sec. 3.3 "FP32-to-FP16 Two-Component Representation", Eq. fp16_high_low;
- *  Sec. 4.2 "Residual Scaling Strategy", Eq. sf_bounds; Sec. 4.3, Eq. recover_eqn;
- *  Sec. 4.5 "Elementwise vs. Termwise Accumulation", Eq. elementwise / Eq. termwise).
+ * (paper: Sec. 3.3, the two-component representation, Eq. fp16_high_low; Sec. 4.2, residual
+ *  scaling, Eq. sf_bounds; Sec. 4.3, Eq. recover_eqn; Sec. 4.5, the two accumulation orders,
+ *  Eq. elementwise / Eq. termwise).
  *
  * Conventions shared by every entry point
  *   - All matrices are ROW-MAJOR with a leading dimension counted in elements.
@@ -65,7 +65,7 @@ enum {
 enum {
   /* Length, in k, of a chain accumulated inside the tensor core before it is added, in FP32 with
    * round-to-nearest, to the running sum held in registers (termwise: the hi*hi stream; the
-   * correction stream is carried whole).  Multiple of 64, default 128.  This is the "k-block" g
+   * correction stream is carried whole).  Multiple of 64, default 128.  This is the k-block g
    * of Sec. 4.5 as realised on this hardware.  The tensor core truncates (rounds toward zero)
    * each time it adds a 16-deep group of products to its accumulator; on data of one sign that
    * bias adds up along a chain, about 0.5 ulp per 16 k (measured Frobenius error on U[0,1)
@@ -198,7 +198,7 @@ int sgemm_cube_presplit(sgemm_cube_handle h, int M, int N, int K,
                         int scale_exp, int accumulation_order, void* stream);
 
 /* Plain FP16 x FP16 -> FP32 GEMM on the tensor cores, D = A16 B16 (or D += A16 B16 when
- * accumulate != 0): one pass of the unfused path, and the "native FP16 GEMM" the paper
+ * accumulate != 0): one pass of the unfused path, and the plain FP16 GEMM the paper
  * contrasts with (Sec. 6.2).
  *   A16_dev M x K FP16 (lda16 >= K), B16_dev K x N FP16 (ldb16 >= N), D_dev M x N FP32 (ldd >= N).
  * Alignment as sgemm_cube_presplit.  Errors as sgemm_cube. */
@@ -258,8 +258,8 @@ int sgemm_cube_exponent_window(sgemm_cube_handle h, int rows, int cols,
                                const float* X_dev, int64_t ldx,
                                int64_t* window_out, void* stream);
 
-/* Residual-overflow detection (paper Sec. 4.2, Rule 2: "... unless residual overflow is explicitly
- * detected and handled"): the number of entries of a split operand whose high word is finite
+/* Residual-overflow detection (paper Sec. 4.2, Rule 2, which allows a larger scale only if
+ * overflowing residuals are caught): the number of entries of a split operand whose high word is finite
  * while its scaled residual word is inf or NaN, i.e. for which (x - hi) 2^s left the FP16 range
  * (the paper's example: x = 32784 at s_b = 12).  A non-zero count means the chosen scale exponent
  * is too large for this operand; sgemm_cube_choose_scale_exp gives one that cannot overflow.
@@ -272,8 +272,8 @@ int sgemm_cube_residual_overflow_count(sgemm_cube_handle h, int rows, int cols,
                                        int64_t* count_out, void* stream);
 
 /* Scale exponent for a pair of operands from their exponent windows (host arithmetic only).
- * Eq. sf_bounds:  -3 - e_min <= s_b <= 26 - e_max  over both operands; following Sec. 4.2 ("scale
- * the residual as far from the underflow threshold as the largest entry permits") the upper end
+ * Eq. sf_bounds:  -3 - e_min <= s_b <= 26 - e_max  over both operands; Sec. 4.2 advises moving
+ * the residuals as far above the underflow threshold as the largest entry allows, so the upper end
  * is taken, capped at 15:  *scale_exp_out = min(26 - e_max, 15).  Full normal FP16 range
  * (e_max = 15) gives 11, e_max <= 14 gives at least 12.
  * *protected_out (optional) = 1 if that value also satisfies the lower end and no high word is

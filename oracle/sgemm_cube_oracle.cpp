@@ -15,7 +15,7 @@
 //        elementwise  [Eq. elementwise]  the three block products folded into one accumulator
 //        reordered elementwise [Sec. 4.5, last paragraph]  corrections of a block summed first
 //   * references: FP64 GEMM, |A||B| in FP64, sequential FP32 GEMM of the unsplit inputs,
-//     and the hi*hi product alone ("native FP16 GEMM" contrast)    [Sec. 6.1, 6.2]
+//     and the hi*hi product alone (the plain FP16 GEMM contrast)    [Sec. 6.1, 6.2]
 //
 // Pins (see tests/test_oracle_*.py): the worked example V = 32784 [Sec. 4.2], the residual-class
 // probability table [Sec. 4.1], Eq. split_error / split_ineqs / ll_bound / main_bound, an
@@ -40,7 +40,7 @@ inline uint32_t f32_bits(float x) { uint32_t w; std::memcpy(&w, &x, 4); return w
 inline float bits_f32(uint32_t w) { float x; std::memcpy(&x, &w, 4); return x; }
 
 // fl16(x): FP32 bit pattern -> FP16 bit pattern, round-to-nearest, ties-to-even.
-// [Sec. 3.3: "This decomposition follows the round-to-nearest-even (RN) rule"; Sec. 4.1 for
+// [Sec. 3.3 fixes round-to-nearest-even for the decomposition; Sec. 4.1 for
 //  the subnormal range: results below 2^-25 round to zero, the midpoint by ties-to-even.]
 uint16_t f16_rn(uint32_t w) {
   const uint16_t sign = (uint16_t)((w >> 16) & 0x8000u);

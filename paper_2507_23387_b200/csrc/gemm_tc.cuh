@@ -1,7 +1,7 @@
 // The tensor-core kernels of the library, one template:
 //
-//   <NTERMS = 1, FUSED = false> : D (+)= A16 * B16       one pass of the unfused path (Sec. 5.4:
-//                                                        "one pipeline instance per term")
+//   <NTERMS = 1, FUSED = false> : D (+)= A16 * B16       one pass of the unfused path (Sec. 5.4
+//                                                        runs each product through its own pipeline)
 //   <NTERMS = 3, FUSED = false> : C = hi_A hi_B + 2^-s (lo_A hi_B + hi_A lo_B) from FP16 words that
 //                                 were split beforehand: all three products of Eq. recover_eqn
 //   <NTERMS = 3, FUSED = true>  : the same from the FP32 operands: converter warps split them on
@@ -14,11 +14,13 @@
 //                round-to-nearest into running sums held in registers, form C, store it
 //   not FUSED (384 threads): warp 8 = TMA producer (FP16 tiles global -> shared, swizzled UMMA
 //                layout), warp 9 = MMA issuer
-//   FUSED (512 threads): warp 13 = TMA producer staging FP32 tiles of A and B in a shared-memory
-//                ring (128-byte swizzle); warps 8-11 = converter warps: FP32 ring -> registers ->
-//                (hi, lo) FP16 words -> the FP16 ring, written directly in the swizzled UMMA
-//                layout; warp 12 = MMA issuer.  Every converter thread works on the same tile
-//                positions in every stage, so its shared-memory offsets are constants.
+//   FUSED (512 threads): warp 13 = TMA producer: FP32 tiles of A and B global -> shared (128-byte
+//                swizzle) into a ring of stages; warps 8-11 = converter warps: each FP32 stage is
+//                split IN PLACE into (hi, lo) FP16 words laid out as swizzled UMMA atoms (every
+//                converter thread works on the same positions of every stage, so its offsets are
+//                constants); warps 14-15 = relay threads: the generic -> async proxy fence and, in
+//                a CTA pair, the arrival on the leader's barrier, kept off the converter warps;
+//                warp 12 = MMA issuer.
 //   The MMA issuer is one thread issuing tcgen05.mma kind::f16 (M = 128, N = 256, K = 16).
 //
 // Why the running sums live in registers.  The tensor core adds products into its FP32
@@ -136,9 +138,10 @@ struct TcGemmParams {
 #endif
 template <int NTERMS, bool PAIR = false, bool FUSED = false>
 struct TcCfg {
-  // k per pipeline stage: 64 for one product; for three products 32 when the converter warps fill
-  // the stages, SGC_BK3 (64, 32 or 16) when TMA does: 64 gives two 96 KB stages (three 64 KB ones
-  // for CTA pairs) and measured 1-3 % faster than four stages of 32 across sizes; 16 much slower
+  // k per pipeline stage: 64 for one product; for three products 32 in the fused kernel (FP32
+  // stages: six of 32 KB for CTA pairs, four of 48 KB for single CTAs), SGC_BK3 (64, 32 or 16) when
+  // TMA loads FP16 words: 64 gives two 96 KB stages (three 64 KB ones for CTA pairs) and measured
+  // 1-3 % faster than four stages of 32 across sizes; 16 much slower
   static constexpr int BK = (NTERMS == 1) ? 64 : (FUSED ? 32 : SGC_BK3);
   static constexpr int BN_CTA = PAIR ? kBN / 2 : kBN;     // B columns held by one CTA
   static constexpr int A_ROW_BYTES = BK * 2;              // 128 or 64: also the swizzle span of A
@@ -917,7 +920,7 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA0, const __grid_constant__
     constexpr int kRegions = Cfg::STAGE_BYTES / 1024;             // 32 (pair) or 48
     static_assert(kRegions % NW == 0, "regions per converter warp");
     constexpr int R = kRegions / NW;
-    constexpr int kBatch = SGC_CONV_BATCH;                                     // regions loaded before converting
+    constexpr int kBatch = SGC_CONV_BATCH;                        // regions loaded before converting
     static_assert(R % kBatch == 0, "batches");
     const int cw = warp - kNumEpiWarps;
     const int ar = lane >> 2, aq = lane & 3;

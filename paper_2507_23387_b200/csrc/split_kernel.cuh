@@ -133,7 +133,7 @@ split_scalar_kernel(int rows, int cols, const float* __restrict__ X, long long l
   }
 }
 
-// C = D_hh + 2^-s * D_x  (the "two final FP32 additions" of the termwise order, Sec. 4.4; the
+// C = D_hh + 2^-s * D_x  (the termwise order ends with two FP32 additions, Sec. 4.4; the
 // first of them, lo*hi + hi*lo, has already happened when D_x was accumulated).
 __global__ void __launch_bounds__(256)
 combine_kernel(int rows, int cols, const float* __restrict__ Dhh, const float* __restrict__ Dx,
@@ -243,7 +243,7 @@ scale_pow2_kernel(int rows, int cols, float* __restrict__ C, long long ldc, int 
   }
 }
 
-// Residual-overflow detection (the "explicitly detected" alternative of Rule 2, Sec. 4.2): counts
+// Residual-overflow detection (Rule 2 of Sec. 4.2 allows a larger scale if overflowing residuals are caught): counts
 // the entries whose high word is finite while the scaled residual is not, i.e. entries for which
 // (x - hi) * 2^s left the FP16 range (the worked example of Sec. 4.2: x = 32784, s = 12).
 // out[0] += count.  HBM-bound: 4 bytes read per element.

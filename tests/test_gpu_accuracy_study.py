@@ -92,3 +92,24 @@ def test_adversarial_sweep_stays_inside_the_componentwise_bound(handle):
     # four-term variant removes it
     r = by["coherent residuals k=16"]
     assert r["termwise_eta"] - r["four_term_eta"] > 2.0
+
+
+def test_harness_componentwise_errors_agree_with_the_oracle_helpers(handle):
+    """The adversarial sweep reports max |C - C64| / (|A||B|) computed with torch FP64 products on the
+    device; the same quantity from the oracle's FP64 reference and its (hand-pinned)
+    componentwise_err on the same inputs must agree, so the harness's tables are tied to the oracle."""
+    mn, K = 128, 256
+    rows = accuracy_study.adversarial_sweep(handle, mn=mn, seeds=1, cancellations=(2.0 ** -6,),
+                                            k_cancel=K, ks_coherent=(64,))
+    by = {r["case"]: r for r in rows}
+    cases = {"cancel c=2^-6": inputs.cancellation_pair(0, mn, mn, K, 2.0 ** -6),
+             "coherent residuals k=64": (inputs.coherent_residuals(0, (mn, 64), 0),
+                                         inputs.coherent_residuals(0, (64, mn), 1))}
+    for name, (A, B) in cases.items():
+        C64, AB = oracle.dgemm_ref(A, B)
+        C = torch.empty((mn, mn), device="cuda:0")
+        for mname, order in (("termwise", binding.TERMWISE), ("elementwise", binding.ELEMENTWISE)):
+            handle.sgemm_cube(torch.from_numpy(A).cuda(), torch.from_numpy(B).cuda(), C, 11, order)
+            want = oracle.componentwise_err(C.cpu().numpy(), C64, AB) * 2.0 ** 24
+            got = by[name][mname + "_eta"]
+            assert abs(got - want) <= 1e-6 * max(want, 1.0), (name, mname, got, want)

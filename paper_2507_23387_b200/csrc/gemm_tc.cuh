@@ -49,9 +49,6 @@ constexpr int kBM = 128;            // CTA tile rows  (UMMA M)
 constexpr int kBN = 256;            // CTA tile cols  (UMMA N)
 constexpr int kNumEpiWarps = 8;     // warps 0-7
 constexpr int kTcThreads = 384;     // not FUSED: + TMA warp + MMA warp (+ 2 idle warps: whole warpgroup)
-#ifndef SGC_RELAY_ARRIVE
-#define SGC_RELAY_ARRIVE 1
-#endif
 // FUSED register split between the accumulate warps and the rest (512 threads x 128 registers),
 // columns per TMEM load in the accumulate warps, regions a converter warp loads before converting
 #ifndef SGC_FUSED_EPI_REGS
@@ -107,12 +104,7 @@ struct TcGemmParams {
   int kchunk_blocks;    // k-block length in units of the stage depth BK
   float inv_scale;      // 2^-s
   unsigned int* err;    // device error word
-  // FUSED only: the FP32 operands (row-major, 16-byte aligned, leading dimensions % 4 == 0)
-  const float* A32;
-  long long lda32;
-  const float* B32;
-  long long ldb32;
-  float scale;          // 2^s
+  float scale;          // FUSED only: 2^s (the FP32 operands themselves come through the tensor maps)
   // Split-K (not FUSED, NTERMS == 3): the k range is cut into `ksplit` slices of `kslice_blocks`
   // stages (a multiple of kchunk_blocks); unit u = slice * tiles + tile writes its hi*hi sums to
   // Phh + slice * pstride and, termwise, its raw correction sums to Px + slice * pstride (both
@@ -735,7 +727,7 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA0, const __grid_constant__
             return true;
           };
           int kb = kb_begin;
-          // stages whose correction products go first (96 or 64 k-steps' worth)
+          // stages whose correction products go first (64 k-steps' worth)
 #ifdef SGC_KLOOK
           constexpr int kLook = SGC_KLOOK;
 #else
@@ -997,13 +989,9 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA0, const __grid_constant__
         SGC_T0();
         fence_proxy_async_smem();
         if (!PAIR || leader) mbar_arrive(&full_bar[s]);
-#if SGC_RELAY_ARRIVE == 0
-        else mbar_arrive_cluster(mapa_u32(smem_u32(&full_bar[s]), 0));   // the leader's barrier
-#elif SGC_RELAY_ARRIVE == 1
+        // remote arrival with the default (CTA-scope) release: what it publishes was made visible
+        // to the async proxy by the fence above, before the arrive was issued
         else mbar_arrive_remote_cta(mapa_u32(smem_u32(&full_bar[s]), 0));
-#else
-        else mbar_arrive_cluster_relaxed(mapa_u32(smem_u32(&full_bar[s]), 0));
-#endif
         SGC_TADD(12, blockIdx.x == 1 && rw == 0);
         SGC_TADD(13, blockIdx.x == 0 && rw == 0);
       }

@@ -241,11 +241,6 @@ __device__ __forceinline__ uint32_t mapa_u32(uint32_t smem_addr, uint32_t rank) 
   asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(smem_addr), "r"(rank));
   return r;
 }
-// Arrive (release at cluster scope) on an mbarrier given by its shared::cluster address.
-__device__ __forceinline__ void mbar_arrive_cluster(uint32_t cluster_addr) {
-  asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" ::"r"(cluster_addr)
-               : "memory");
-}
 // Arrive on a remote mbarrier with the default semantics (release at CTA scope).
 __device__ __forceinline__ void mbar_arrive_remote_cta(uint32_t cluster_addr) {
   asm volatile("mbarrier.arrive.shared::cluster.b64 _, [%0];" ::"r"(cluster_addr) : "memory");
@@ -289,14 +284,6 @@ __device__ __forceinline__ bool mbar_wait_bounded_cluster(uint64_t* bar, uint32_
       return false;
     }
   }
-}
-__device__ __forceinline__ void fence_proxy_async_all() {
-  asm volatile("fence.proxy.async;" ::: "memory");
-}
-// Generic-proxy writes to shared memory made visible to the async proxy of every CTA of the
-// cluster (in a CTA pair the peer's tensor core reads this CTA's half of the B tile).
-__device__ __forceinline__ void fence_proxy_async_smem_cluster() {
-  asm volatile("fence.proxy.async.shared::cluster;" ::: "memory");
 }
 // 2-D tiled load into this CTA's shared memory whose completion bytes are counted on the
 // mbarrier at the same offset in the LEADER CTA (bit 24 of a shared::cluster address holds the

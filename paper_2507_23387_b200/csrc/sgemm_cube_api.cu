@@ -123,10 +123,10 @@ int set_kernel_attrs(sgemm_cube_ctx* h) {
 }
 
 // 2-CTA clusters (each CTA loads half of the B tile: two thirds of the L2 -> SM traffic of single
-// CTAs) measured faster than single CTAs for the TMA-fed kernels from 512^3 up (e.g. 4096^3: 407
-// against 378, 8192^3: 458 against 439 TFLOP/s); by default they are used whenever the problem has
-// more than one 128-row block.  The converter-fed kernel is slower in pairs (172 against 193) and
-// only uses them when asked to.
+// CTAs, and two thirds of the tensor core's shared-memory reads) measured faster than single CTAs
+// from 512^3 up (e.g. 8192^3: 458 against 439 TFLOP/s from FP16 words, 374 against 270 for the
+// fused converter kernel); by default they are used whenever the problem has more than one 128-row
+// block.
 bool use_pair(const sgemm_cube_ctx* h, int M, int N, bool fused) {
   (void)N;
   (void)fused;
@@ -301,7 +301,7 @@ int launch_tc_gemm(sgemm_cube_ctx* h, int M, int N, int K, const uint16_t* Ahi, 
   if (p.kchunk_blocks < 1) p.kchunk_blocks = 1;
   p.inv_scale = inv_scale;
   p.err = h->err_dev;
-  p.A32 = nullptr; p.lda32 = 0; p.B32 = nullptr; p.ldb32 = 0; p.scale = 1.f;
+  p.scale = 1.f;
   p.ksplit = 1; p.kslice_blocks = 0; p.Phh = nullptr; p.Px = nullptr; p.pstride = 0; p.ldp = 0;
   p.kclock = (NTERMS == 3 && h->time_kernel && h->err_dev_has_clock)
                  ? reinterpret_cast<unsigned long long*>(h->err_dev + 16) : nullptr;
@@ -383,8 +383,6 @@ int launch_fused(sgemm_cube_ctx* h, int M, int N, int K, const float* A, int64_t
   if (p.kchunk_blocks < 1) p.kchunk_blocks = 1;
   p.inv_scale = ldexpf(1.0f, -s);
   p.err = h->err_dev;
-  p.A32 = A; p.lda32 = lda;
-  p.B32 = B; p.ldb32 = ldb;
   p.scale = ldexpf(1.0f, s);
   p.ksplit = 1; p.kslice_blocks = 0; p.Phh = nullptr; p.Px = nullptr; p.pstride = 0; p.ldp = 0;
   p.kclock = (h->time_kernel && h->err_dev_has_clock)
@@ -434,9 +432,9 @@ int launch_two_phase(sgemm_cube_ctx* h, int M, int N, int K, const float* A, int
 }
 
 // The entry point's strategy choice.  The fused kernel re-splits every operand tile once per
-// output tile and has to pull FP32 tiles (twice the bytes of the FP16 words) through L2 for each
-// of them, which bounds it well below the tensor-core rate on large problems; there the split is
-// done once up front.  Small problems keep the single launch.
+// output tile, and its staging and conversion traffic shares the shared-memory pipe with the
+// tensor core's operand reads, which keeps the tensor pipe about 60 % busy on large problems
+// against 90 % when the split is done once up front.  Small problems keep the single launch.
 int launch_sgemm_cube(sgemm_cube_ctx* h, int M, int N, int K, const float* A, int64_t lda, const float* B,
                       int64_t ldb, float* C, int64_t ldc, int s, int order, cudaStream_t st) {
   bool two_phase = (h->strategy == 2) ||

@@ -35,6 +35,8 @@
 //   NTERMS == 1             : the regions alternate between consecutive k-blocks (double buffer)
 //   NTERMS == 3 termwise    : R0 = hi*hi partial of the current k-block, R1 = correction stream
 //   NTERMS == 3 elementwise : R0 = hi*hi partial, R1 = correction partial of the current k-block
+//   NTERMS == 3 reordered elementwise, s <= 15: each k-block's value P_x / s_f + P_hh is formed in
+//                             one region (scale-d MMA, see reord_fast); the regions alternate
 #pragma once
 
 #include <cuda_fp16.h>
@@ -404,6 +406,13 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA0, const __grid_constant__
     kb1 = (ksplit > 1) ? min(num_kb, kb0 + p.kslice_blocks) : num_kb;
   };
   const int chunk = p.kchunk_blocks;                           // stages per k-block g
+  // Reordered elementwise order, fast form: a k-block's value P_x / s_f + P_hh is formed inside one
+  // TMEM region (the correction products first, then the first hi*hi MMA scales the accumulator
+  // by 2^-s as it adds: tcgen05.mma's scale-d operand), so the accumulate warps read one region per
+  // block and the two regions alternate between blocks: block g + 1 accumulates while block g is
+  // read.  Needs s <= 15 (the instruction's range) and all stages of a block resident at once.
+  const int scale_exp = 127 - (int)((__float_as_uint(p.inv_scale) >> 23) & 0xFFu);
+  const bool reord_fast = REORD && (NTERMS == 3) && scale_exp >= 0 && scale_exp <= 15 && 2 * chunk <= STAGES;
 
   // Register budget when FUSED (512 threads x 128 registers): the accumulate warps hold a
   // 128 x 256 FP32 tile in registers, so warpgroups 2-3 hand registers over to warpgroups 0-1
@@ -457,7 +466,7 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA0, const __grid_constant__
       unit_rc(unit, tm, tn, kb0, kb1, slice);
       const int unit_chunks = (kb1 - kb0 + chunk - 1) / chunk;
       for (int c = 0; c < unit_chunks && ok; ++c, ++gchunk) {
-        const int r_main = (NTERMS == 1) ? (int)(gchunk & 1) : 0;
+        const int r_main = (NTERMS == 1 || reord_fast) ? (int)(gchunk & 1) : 0;
         const bool with_x = (NTERMS == 3) && (p.order == 1);
         constexpr bool reordered = (NTERMS == 3) && REORD;
         {
@@ -469,10 +478,11 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA0, const __grid_constant__
         tc_fence_after_sync();
         const uint32_t t_main = tmem_base + lane_addr + r_main * kBN + half * 128;
         const uint32_t t_x = tmem_base + lane_addr + kBN + half * 128;
-        if constexpr (reordered) {
+        if (reordered && !reord_fast) {
           // Reordered elementwise (Sec. 4.5, last paragraph): the block's corrections, already
           // summed at their own scale, are scaled and added to the block's hi*hi product, and the
-          // accumulator takes the block once:  acc = acc + (P_x / s_f + P_hh).
+          // accumulator takes the block once:  acc = acc + (P_x / s_f + P_hh).  (The fast form
+          // gets the block's value ready-made from one region and takes the plain path below.)
           if (!wait_tfull(1)) { ok = false; break; }
           tc_fence_after_sync();
           constexpr int GR = 16;
@@ -758,6 +768,62 @@ tc_gemm_kernel(const __grid_constant__ CUtensorMap tmA0, const __grid_constant__
             if (release) commit_both(&empty_bar[i % STAGES]);
             return true;
           };
+          if constexpr (REORD && NTERMS == 3) {
+            if (reord_fast) {
+              // One region per k-block, alternating: all correction products of the block first
+              // (from zero), then its hi*hi products, the first of which takes the accumulator
+              // scaled by 2^-s:  D = P_hh + 2^-s P_x.  The order inside each chain is the usual one.
+              const int r = (int)(gchunk & 1);
+              const uint32_t d = tmem_base + r * kBN;
+              if (!wait(&tempty_bar[r], (fills[r] & 1) ^ 1, kErrMmaTmemEmptyWait)) { ok = false; break; }
+              tc_fence_after_sync();
+              const int n = kb_end - kb_begin;
+              constexpr int kMaxN = STAGES / 2 > 0 ? STAGES / 2 : 1;
+              uint32_t stv[kMaxN];
+#pragma unroll
+              for (int l = 0; l < kMaxN; ++l) {
+                if (l < n && ok) {
+                  ok = stage_ready(it + l, stv[l]);
+                  if (ok) {
+                    const uint32_t a_hi = a_desc_lo0 + (stv[l] >> 4), a_lo = a_hi + (Cfg::A_LO_OFF >> 4);
+                    const uint32_t b_hi = b_desc_lo0 + ((stv[l] + Cfg::B_OFF) >> 4);
+                    const uint32_t b_lo = b_hi + (Cfg::B_LO_OFF >> 4);
+                    constexpr int G = (BK < 32 ? BK : 32) / 16;
+#pragma unroll
+                    for (int j0 = 0; j0 < BK / 16; j0 += G) {
+#pragma unroll
+                      for (int j = j0; j < j0 + G; ++j)
+                        mma(d, desc(a_lo + 2 * j, a_desc_hi), desc(b_hi + 128 * j, b_desc_hi),
+                            (l == 0 && j == 0) ? 0u : 1u);
+#pragma unroll
+                      for (int j = j0; j < j0 + G; ++j)
+                        mma(d, desc(a_hi + 2 * j, a_desc_hi), desc(b_lo + 128 * j, b_desc_hi), 1u);
+                    }
+                  }
+                }
+              }
+#pragma unroll
+              for (int l = 0; l < kMaxN; ++l) {
+                if (l < n && ok) {
+                  const uint32_t a_hi = a_desc_lo0 + (stv[l] >> 4);
+                  const uint32_t b_hi = b_desc_lo0 + ((stv[l] + Cfg::B_OFF) >> 4);
+#pragma unroll
+                  for (int j = 0; j < BK / 16; ++j) {
+                    const uint64_t da = desc(a_hi + 2 * j, a_desc_hi);
+                    const uint64_t db = desc(b_hi + 128 * j, b_desc_hi);
+                    if (l == 0 && j == 0) umma_f16_ss_scale_d_rt(scale_exp, d, da, db, idesc, PAIR);
+                    else mma(d, da, db, 1u);
+                  }
+                  commit_both(&empty_bar[(it + l) % STAGES]);
+                }
+              }
+              if (!ok) break;
+              commit_both(&tfull_bar[r]);
+              fills[r]++;
+              it += n;
+              continue;
+            }
+          }
           int kb = kb_begin;
           // stages whose correction products go first (64 k-steps' worth)
 #ifdef SGC_KLOOK

@@ -176,6 +176,46 @@ __device__ __forceinline__ void umma_f16_ss(uint32_t d_tmem, uint64_t a_desc, ui
       : "memory");
 }
 
+// D[tmem] = A[smem] * B[smem] + D[tmem] * 2^-SCALE  (kind::f16 on sm_100a; SCALE = 0..15 is an
+// immediate of the instruction): the accumulator is scaled down by a power of two before the
+// products are added.
+template <int SCALE>
+__device__ __forceinline__ void umma_f16_ss_scale_d(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc,
+                                                    uint32_t idesc, bool pair) {
+  if (pair) {
+    asm volatile(
+        "{\n"
+        ".reg .pred p;\n"
+        "setp.ne.b32 p, 1, 0;\n"
+        "tcgen05.mma.cta_group::2.kind::f16 [%0], %1, %2, %3, p, %4;\n"
+        "}\n"
+        ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "n"(SCALE)
+        : "memory");
+  } else {
+    asm volatile(
+        "{\n"
+        ".reg .pred p;\n"
+        "setp.ne.b32 p, 1, 0;\n"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p, %4;\n"
+        "}\n"
+        ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "n"(SCALE)
+        : "memory");
+  }
+}
+// The same with the scale chosen at run time (a switch over the 16 instruction forms).
+__device__ __forceinline__ void umma_f16_ss_scale_d_rt(int scale, uint32_t d_tmem, uint64_t a_desc,
+                                                       uint64_t b_desc, uint32_t idesc, bool pair) {
+  switch (scale) {
+#define SGC_SCALE_CASE(n) case n: umma_f16_ss_scale_d<n>(d_tmem, a_desc, b_desc, idesc, pair); break;
+    SGC_SCALE_CASE(0) SGC_SCALE_CASE(1) SGC_SCALE_CASE(2) SGC_SCALE_CASE(3) SGC_SCALE_CASE(4)
+    SGC_SCALE_CASE(5) SGC_SCALE_CASE(6) SGC_SCALE_CASE(7) SGC_SCALE_CASE(8) SGC_SCALE_CASE(9)
+    SGC_SCALE_CASE(10) SGC_SCALE_CASE(11) SGC_SCALE_CASE(12) SGC_SCALE_CASE(13) SGC_SCALE_CASE(14)
+    SGC_SCALE_CASE(15)
+#undef SGC_SCALE_CASE
+    default: break;
+  }
+}
+
 // Arrive on an mbarrier once all tcgen05 operations issued so far by this thread have completed
 // (implies tcgen05.fence::before_thread_sync).
 __device__ __forceinline__ void umma_commit(uint64_t* bar) {

@@ -489,6 +489,29 @@ def test_reordered_elementwise_order(handle, path, shape):
     gates(run(handle, path, padded_dev(A2, 4), padded_dev(B2, 4), 11, R), A2, B2, 11, R, label="nonneg")
 
 
+@pytest.mark.parametrize("path", ["fused", "two_phase"])
+@pytest.mark.parametrize("s,kblock", [(15, 64), (16, 64), (11, 256), (0, 64)])
+def test_reordered_elementwise_both_forms_of_the_kernel(handle, path, s, kblock):
+    """The reordered order has two realisations in the kernel: for s <= 15 and k-blocks short enough
+    to be resident at once, a block's value P_x / s_f + P_hh is formed inside one accumulator (the
+    first hi*hi MMA scales the accumulator by 2^-s as it adds) and the two accumulators alternate
+    between blocks; otherwise both partial sums are read and combined in registers.  Same order of
+    Sec. 4.5 (last paragraph), same gates, for scale exponents and k-blocks on both sides."""
+    M, N, K = 300, 520, 1000
+    A, B = inputs.make_pair("exponent_spread", 5, M, N, K)
+    if s == 0:
+        A, B = inputs.make_pair("uniform_pm1", 5, M, N, K)
+    try:
+        handle.sgemm_cube_set_option(binding.OPT_ELEMENTWISE_K_BLOCK, kblock)
+        for pair in (1, 0):
+            handle.sgemm_cube_set_option(binding.OPT_CTA_PAIR, pair)
+            C = run(handle, path, padded_dev(A, 4), padded_dev(B, 4), s, R)
+            gates(C, A, B, s, R, kb=kblock, label="reordered %s s=%d kblock=%d pair=%d" % (path, s, kblock, pair))
+    finally:
+        handle.sgemm_cube_set_option(binding.OPT_CTA_PAIR, 2)
+        handle.sgemm_cube_set_option(binding.OPT_ELEMENTWISE_K_BLOCK, K_BLOCK[R])
+
+
 def test_reordered_elementwise_keeps_what_a_block_adds_up_to(handle):
     # Block 0 makes the accumulator 2^10 (ulp 2^-13).  Block 1 holds hi*hi = 2^-14 (1 - 2^-20),
     # just under half an ulp, and a correction of 2^-29: added one after the other to the

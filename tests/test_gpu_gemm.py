@@ -164,6 +164,44 @@ def test_strategies_agree_bitwise(handle):
         assert np.array_equal(C1, C2) and np.array_equal(C1, C3)
 
 
+@pytest.mark.parametrize("s", [0, 5, 15, 16, 20, 24])
+def test_in_kernel_split_matches_the_split_kernel_for_every_scale_exponent(handle, s):
+    """The converter warps have two forms of the split arithmetic (s <= 15: packed multiply and
+    mixed-precision FMA; s > 15: subtract and multiply), the split kernel has one; whatever the scale
+    exponent, and also on entries outside the method's comfortable range (FP16-subnormal high words,
+    values near the top of the FP16 range, signed zeros), the fused kernel must produce the bits of
+    the two-phase route.  Values are chosen so that nothing overflows to inf at the largest s
+    (where one form gives inf and the other NaN)."""
+    rng = np.random.default_rng(11 + s)
+    M, N, K = 260, 520, 200
+    if s <= 16:          # Rule 2 of Sec. 4.2: s <= 26 - e_max, and these inputs have e_max = 10
+        A = inputs.exponent_spread(21, (M, K), stream=0)
+        B = inputs.exponent_spread(21, (K, N), stream=1)
+    else:                # |x| < 1: residuals stay in range up to s = 24
+        A, B = inputs.make_pair("uniform_pm1", 21, M, N, K)
+    # a few rows / columns of awkward values
+    A[3, :] = (rng.standard_normal(K) * 2.0 ** -22).astype(np.float32)        # hi subnormal in FP16
+    A[7, :] = 0.0
+    A[9, ::2] = -0.0
+    B[:, 5] = (rng.standard_normal(K) * 2.0 ** -17).astype(np.float32)
+    if s <= 11:
+        A[11, :] = (rng.uniform(20000, 60000, K) * rng.choice([-1, 1], K)).astype(np.float32)
+    for order in (T, E, binding.ELEMENTWISE_REORDERED):
+        ref = None
+        for path in ("two_phase", "fused"):
+            for pair in (1, 0):
+                handle.sgemm_cube_set_option(binding.OPT_CTA_PAIR, pair)
+                try:
+                    C = run(handle, path, to_dev(A), to_dev(B), s, order)
+                finally:
+                    handle.sgemm_cube_set_option(binding.OPT_CTA_PAIR, 2)
+                assert np.isfinite(C).all()
+                if ref is None:
+                    ref = C
+                else:
+                    assert np.array_equal(C, ref), (s, order, path, pair)
+
+
 @pytest.mark.parametrize("n", [4096, 8192])
 def test_strategies_and_cta_modes_agree_on_the_full_matrix(handle, n):
     """Several waves of the persistent grid, the partly filled last wave included: the fused
